@@ -1,0 +1,176 @@
+/*
+ * d3.h -- C ABI of libd3: Position-Aware Depth Decay Decoding (D3) on one GPU.
+ *
+ * The library runs the autoregressive decode step of a Llama-style decoder in
+ * which generated token T_i executes only floor(L * alpha^i) decoder blocks
+ * (paper: Abstract; Sec. 3.4).  The dropped blocks form one window that opens
+ * at the "flex layer" start id (Appendix, Table "HP description"); a token's
+ * hidden state passes through dropped blocks unchanged and the KV-cache
+ * entries of dropped blocks are filled per `kv_fill` (Sec. 1 (i); Sec. 3.2).
+ *
+ * Conventions
+ *  - Every function returns D3_OK (0) or a negative D3_E* code; nothing throws,
+ *    aborts or traps.  Arguments are validated on the host before any launch;
+ *    a call that fails validation changes no state.
+ *  - Pointers are HOST pointers unless the name ends in `_dev`.
+ *  - The caller allocates and owns all device memory (weights, KV cache,
+ *    scratch, logits) and the CUDA stream; the library allocates no device
+ *    memory, never copies weights, and borrows the pointers until d3_free.
+ *  - Work is enqueued on the stream given to d3_load and is asynchronous;
+ *    d3_sync waits for it.  A model is not thread-safe.
+ *  - Weights are bf16, row-major [out][in].  Activations, accumulators, the
+ *    residual stream and logits are fp32.  The KV cache is bf16.
+ */
+#ifndef D3_H_
+#define D3_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define D3_OK 0
+#define D3_EINVAL (-1)    /* bad argument (null, out of range, NaN, unsupported size) */
+#define D3_ECAPACITY (-2) /* a sequence would exceed max_seq, or batch > max_batch     */
+#define D3_ESTATE (-3)    /* decode on a slot never prefilled; a slot twice in a batch */
+#define D3_ECUDA (-4)     /* a CUDA runtime call failed                                */
+#define D3_ETIMEOUT (-5)  /* a bounded device-side wait ran out                         */
+
+#define D3_MAX_BATCH 64   /* rows per step                                             */
+#define D3_MAX_LAYERS 128
+
+/* Which blocks a token with retained count n drops. */
+#define D3_ANCHOR_START 0 /* [start_id, start_id + L - n), n = max(floor(L alpha^i), start_id):
+                             the paper's rule (Appendix, Table "HP description")      */
+#define D3_ANCHOR_TAIL 1  /* [n, L): the Early-Exit direction (Sec. 1 (ii))           */
+
+/* What is written to the KV cache of a dropped block for the token (Sec. 3.2). */
+#define D3_FILL_NONE 0      /* nothing                                                 */
+#define D3_FILL_COPY 1      /* the token's K,V of the block just below the window
+                               (zeros when the window opens at block 0)               */
+#define D3_FILL_RECOMPUTE 2 /* the dropped block's own norm, W_k, W_v and RoPE applied
+                               to the carried hidden state                            */
+
+#define D3_KV_CONTIGUOUS 0  /* K then V, each [L][slot][Hkv][max_seq][head_dim] bf16  */
+
+typedef struct d3_config {
+  uint32_t struct_size;     /* sizeof(d3_config), checked                              */
+  int32_t n_layers;         /* L, 1..D3_MAX_LAYERS                                     */
+  int32_t d_model;          /* multiple of 8                                           */
+  int32_t n_q_heads;
+  int32_t n_kv_heads;       /* divides n_q_heads (grouped-query attention)             */
+  int32_t head_dim;         /* 32, 64 or 128                                           */
+  int32_t d_ffn;            /* multiple of 8                                           */
+  int32_t vocab;
+  float rms_eps;
+  float rope_base;
+  int32_t max_slots;        /* sequences the KV cache holds                            */
+  int32_t max_seq;          /* positions per sequence                                  */
+  int32_t max_batch;        /* rows per decode step, 1..D3_MAX_BATCH                   */
+  int32_t start_id;         /* 0..L: first droppable block, 0-based (floor(start * L)) */
+  int32_t anchor;           /* D3_ANCHOR_*                                             */
+  int32_t kv_fill;          /* D3_FILL_*                                               */
+  int32_t kv_layout;        /* D3_KV_CONTIGUOUS                                        */
+} d3_config;
+
+/* DEVICE pointers to bf16 tensors; the per-layer members are HOST arrays of L
+ * device pointers.  Every tensor must be 16-byte aligned.
+ *   embed, lm_head [vocab][d];  *_norm [d] gains;
+ *   wqkv [(Hq + 2 Hkv) * head_dim][d]: rows of W_q, then W_k, then W_v;
+ *   wo [d][Hq * head_dim];  w_gate, w_up [f][d];  w_down [d][f].            */
+typedef struct d3_weights {
+  const void *embed_dev, *lm_head_dev, *final_norm_dev;
+  const void *const *attn_norm_dev;
+  const void *const *wqkv_dev;
+  const void *const *wo_dev;
+  const void *const *mlp_norm_dev;
+  const void *const *w_gate_dev;
+  const void *const *w_up_dev;
+  const void *const *w_down_dev;
+} d3_weights;
+
+/* What one decode step did (all integers exact).  `n` and `m_per_layer` are
+ * caller-provided HOST arrays of `batch` and L entries, or NULL. */
+typedef struct d3_step_stats {
+  int32_t *n;                /* retained block count of each row, caller order        */
+  int32_t *m_per_layer;      /* rows that executed each block                          */
+  int64_t rows_layers;       /* sum of m_per_layer == sum of n                         */
+  int32_t layers_touched;    /* blocks executed by at least one row                    */
+  int32_t kernel_launches;   /* kernels this step enqueued                             */
+  int64_t algorithmic_bytes; /* weights of touched blocks + KV read by retained blocks
+                                + KV written + LM head + embedding rows + logits out  */
+} d3_step_stats;
+
+typedef struct d3_model d3_model;
+
+/* floor(L * alpha^i): blocks retained when generating T_i (Abstract; Sec. 3.4).
+ * Host, pure.  alpha in (0, 1], i >= 0, 0 <= L; otherwise D3_EINVAL. */
+int32_t d3_depth(int32_t L, double alpha, int64_t i);
+
+/* The batch schedule of one step (Sec. 3.4 + Appendix Table "HP description";
+ * batching: Sec. 3.1).  Host, pure; the same integers the device kernel derives.
+ * For each of `batch` rows with generation index gen_index[b]: retained count
+ * n[b], dropped window [lo[b], hi[b]); perm = rows ordered by n descending,
+ * ties by row index; m_per_layer[l] = rows that run block l (always a prefix of
+ * perm).  Output arrays are caller-owned; rows_layers / layers_touched may be NULL. */
+int32_t d3_schedule(int32_t L, double alpha, int32_t start_id, int32_t anchor, int32_t batch,
+                    const int32_t *gen_index, int32_t *n, int32_t *lo, int32_t *hi,
+                    int32_t *perm, int32_t *m_per_layer, int64_t *rows_layers,
+                    int32_t *layers_touched);
+
+/* Bytes of KV cache and of scratch the caller must allocate for `cfg`
+ * (256-byte aligned device buffers). */
+int32_t d3_workspace_bytes(const d3_config *cfg, size_t *kv_bytes, size_t *scratch_bytes);
+
+/* Create a model over caller-owned device memory.  Enqueues one set-up kernel
+ * (rotary table) on `cuda_stream` (a cudaStream_t passed as void*; NULL = the
+ * default stream).  The KV cache is not cleared. */
+int32_t d3_load(const d3_config *cfg, const d3_weights *weights, void *kv_dev, void *scratch_dev,
+                void *cuda_stream, d3_model **out);
+
+/* Initiation phase (Sec. 3.1; Sec. 4.1: prompts pass through all blocks): run
+ * every prompt token through all L blocks, fill the slot's cache from position
+ * 0, and write the logits that choose T_0 to logits_dev [vocab] (fp32; may be
+ * NULL).  Resets the slot first. */
+int32_t d3_prefill(d3_model *m, int32_t slot, const int32_t *tokens, int32_t n_tokens,
+                   float *logits_dev);
+
+/* Generation phase, one step (Sec. 3.4).  Row b feeds tokens[b] = T_{i-1} of the
+ * sequence in slots[b] at the slot's next cache position, with i = gen_index[b]
+ * >= 1 the index of the token being generated; it runs the blocks outside its
+ * window and receives logits_dev[b][vocab] (fp32, caller row order), the
+ * logits that choose T_i.  alpha in (0, 1] applies to this call.  `stats` may
+ * be NULL.  Slots must be distinct and prefilled.
+ * tokens_dev (nullable): when given, int32 [batch] DEVICE token ids that
+ * replace `tokens` (which may then be NULL), so that a greedy loop can feed
+ * d3_argmax's output back without a host round trip. */
+int32_t d3_decode_step(d3_model *m, int32_t batch, const int32_t *slots, const int32_t *tokens,
+                       const int32_t *gen_index, double alpha, float *logits_dev,
+                       d3_step_stats *stats, const int32_t *tokens_dev);
+
+/* argmax over each row of logits_dev [batch][vocab], lowest index on ties
+ * (greedy choice: Sec. 3.2, footnote on lm_head) -> tokens_dev [batch] int32. */
+int32_t d3_argmax(d3_model *m, const float *logits_dev, int32_t batch, int32_t *tokens_dev);
+
+/* Diagnostics of the last step, after waiting for the stream:
+ * the device kernel's schedule (each array HOST, nullable: n, perm [batch];
+ * m_per_layer [L]; counters[0] = rows_layers, counters[1] = layers_touched). */
+int32_t d3_read_schedule(d3_model *m, int32_t *n, int32_t *perm, int32_t *m_per_layer,
+                         int64_t *counters);
+/* the residual stream before the final norm, caller row order, to HOST [batch][d] fp32 */
+int32_t d3_read_hidden(d3_model *m, float *hidden);
+/* one KV-cache entry to HOST: k, v [Hkv * head_dim] fp32 */
+int32_t d3_read_kv(d3_model *m, int32_t layer, int32_t slot, int32_t pos, float *k, float *v);
+
+int32_t d3_slot_pos(const d3_model *m, int32_t slot); /* tokens cached; D3_ESTATE if never prefilled */
+int32_t d3_reset_slot(d3_model *m, int32_t slot);
+int32_t d3_sync(d3_model *m); /* wait for the stream; returns a deferred device status */
+void d3_free(d3_model *m);    /* host bookkeeping only */
+const char *d3_strerror(int32_t code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* D3_H_ */

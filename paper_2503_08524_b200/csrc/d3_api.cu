@@ -1,0 +1,482 @@
+// C ABI of libd3: argument validation, host bookkeeping, the host copy of the
+// depth schedule, and the per-step launch sequence.
+#include <math.h>
+#include <string.h>
+
+#include <map>
+#include <new>
+#include <vector>
+
+#include "d3_internal.cuh"
+
+namespace d3 {
+
+static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+Layout make_layout(const d3_config &c) {
+  Layout y;
+  const size_t B = (size_t)c.max_batch;
+  const size_t qkv_rows = (size_t)(c.n_q_heads + 2 * c.n_kv_heads) * c.head_dim;
+  y.max_splits = 32;
+  size_t off = 0;
+  y.sched = off;    off = align_up(off + sizeof(DevSched), 256);
+  y.rope = off;     off = align_up(off + (size_t)c.max_seq * (c.head_dim / 2) * sizeof(float2), 256);
+  y.x = off;        off = align_up(off + B * c.d_model * 4, 256);
+  y.qkv = off;      off = align_up(off + B * qkv_rows * 4, 256);
+  y.attn_out = off; off = align_up(off + B * c.n_q_heads * c.head_dim * 4, 256);
+  y.part_o = off;   off = align_up(off + B * c.n_q_heads * y.max_splits * c.head_dim * 4, 256);
+  y.part_ml = off;  off = align_up(off + B * c.n_q_heads * y.max_splits * 2 * 4, 256);
+  y.u = off;        off = align_up(off + B * c.d_ffn * 4, 256);
+  y.total = off;
+  return y;
+}
+
+static bool config_ok(const d3_config *c) {
+  if (!c || c->struct_size != sizeof(d3_config)) return false;
+  if (c->n_layers < 1 || c->n_layers > D3_MAX_LAYERS) return false;
+  if (c->d_model < 8 || c->d_model % 8) return false;
+  if (c->d_ffn < 8 || c->d_ffn % 8) return false;
+  if (c->n_q_heads < 1 || c->n_kv_heads < 1 || c->n_q_heads % c->n_kv_heads) return false;
+  if (c->head_dim != 32 && c->head_dim != 64 && c->head_dim != 128) return false;
+  if (c->vocab < 1 || c->max_slots < 1 || c->max_seq < 1) return false;
+  if (c->max_batch < 1 || c->max_batch > D3_MAX_BATCH) return false;
+  if (!(c->rms_eps >= 0.f) || !(c->rope_base > 0.f)) return false;
+  if (c->start_id < 0 || c->start_id > c->n_layers) return false;
+  if (c->anchor != D3_ANCHOR_START && c->anchor != D3_ANCHOR_TAIL) return false;
+  if (c->kv_fill < D3_FILL_NONE || c->kv_fill > D3_FILL_RECOMPUTE) return false;
+  if (c->kv_layout != D3_KV_CONTIGUOUS) return false;
+  return true;
+}
+
+static bool alpha_ok(double a) { return a > 0.0 && a <= 1.0; }  // false for NaN
+
+static int32_t depth_host(int32_t L, double alpha, int64_t i) {
+  return (int32_t)floor((double)L * pow(alpha, (double)i));
+}
+
+// thr[n] = smallest i with floor(L alpha^i) < n (n = 1..L); INT32_MAX if none.
+static void thresholds(int32_t L, double alpha, int32_t *thr) {
+  thr[0] = 0;
+  const int64_t imax = 0x7ffffffe;
+  for (int n = 1; n <= L; ++n) {
+    if (depth_host(L, alpha, imax) >= n) { thr[n] = 0x7fffffff; continue; }
+    int64_t lo = 0, hi = imax;  // depth(lo) >= n, depth(hi) < n
+    while (hi - lo > 1) {
+      int64_t mid = lo + (hi - lo) / 2;
+      if (depth_host(L, alpha, mid) >= n) lo = mid; else hi = mid;
+    }
+    thr[n] = (int32_t)hi;
+  }
+}
+
+}  // namespace d3
+
+using namespace d3;
+
+struct d3_model {
+  d3_config cfg;
+  Dims dm;
+  Layout lay;
+  cudaStream_t stream;
+  const bf16 *embed, *lm_head, *final_norm;
+  std::vector<const bf16 *> attn_norm, wqkv, wo, mlp_norm, w_gate, w_up, w_down;
+  bf16 *Kc, *Vc;
+  char *scratch;
+  std::vector<int32_t> pos;  // tokens cached per slot; -1 = never prefilled
+  std::map<uint64_t, std::vector<int32_t>> thr_cache;
+  // last step (diagnostics)
+  int32_t last_B;
+  int32_t last_perm[D3_MAX_BATCH];
+  int64_t layer_bytes, head_bytes;
+
+  DevSched *sched() const { return reinterpret_cast<DevSched *>(scratch + lay.sched); }
+  float2 *rope() const { return reinterpret_cast<float2 *>(scratch + lay.rope); }
+  float *x() const { return reinterpret_cast<float *>(scratch + lay.x); }
+  float *qkv() const { return reinterpret_cast<float *>(scratch + lay.qkv); }
+  float *attn_out() const { return reinterpret_cast<float *>(scratch + lay.attn_out); }
+  float *part_o() const { return reinterpret_cast<float *>(scratch + lay.part_o); }
+  float *part_ml() const { return reinterpret_cast<float *>(scratch + lay.part_ml); }
+  float *u() const { return reinterpret_cast<float *>(scratch + lay.u); }
+};
+
+static const int32_t *thr_for(d3_model *m, double alpha) {
+  uint64_t key;
+  memcpy(&key, &alpha, 8);
+  auto it = m->thr_cache.find(key);
+  if (it == m->thr_cache.end()) {
+    if (m->thr_cache.size() > 64) m->thr_cache.clear();
+    std::vector<int32_t> t(D3_MAX_LAYERS + 1, 0);
+    thresholds(m->cfg.n_layers, alpha, t.data());
+    it = m->thr_cache.emplace(key, std::move(t)).first;
+  }
+  return it->second.data();
+}
+
+// Enqueue one step over the rows described by `a` (already validated).
+// logits_mode: ROWS_ALL -> logits_dev[caller row][V]; ROWS_LAST -> logits_dev[V]
+// for the last row; logits_dev may be NULL (no LM head).
+static int32_t run_step(d3_model *m, const StepArgs &a, const int32_t *n, const int32_t *lo,
+                        const int32_t *hi, const int32_t *perm, const int32_t *m_l,
+                        float *logits_dev, int logits_mode, int32_t *launches_out) {
+  const d3_config &c = m->cfg;
+  const Dims &dm = m->dm;
+  cudaStream_t st = m->stream;
+  const int B = a.B, L = c.n_layers;
+  int launches = 0;
+  launches += launch_schedule_embed(a, m->sched(), m->embed, m->x(), dm.d, st);
+  const int nq = dm.Hq * dm.dh, nkv = dm.Hkv * dm.dh;
+  const int G = dm.Hq / dm.Hkv, GQ = (G % 4 == 0) ? 4 : (G % 2 == 0) ? 2 : 1;
+
+  GemvArgs g;
+  memset(&g, 0, sizeof(g));
+  g.sched = m->sched();
+  g.eps = c.rms_eps;
+  for (int l = 0; l < L; ++l) {
+    const int ml = m_l[l];
+    g.layer = l;
+    if (ml > 0) {
+      // RMSNorm + QKV projection
+      g.row_mode = ROWS_PREFIX;
+      g.W = m->wqkv[l]; g.W2 = nullptr; g.R = dm.qkv_rows; g.K = dm.d;
+      g.act = m->x(); g.act_stride = dm.d; g.gain = m->attn_norm[l];
+      g.out = m->qkv(); g.out_stride = dm.qkv_rows; g.out_col0 = 0;
+      launches += launch_gemv(g, EPI_STORE, ml, st);
+      launches += launch_rope_append(m->qkv(), m->rope(), m->Kc, m->Vc, m->sched(), l, ROWS_PREFIX,
+                                     0, ml, dm, st);
+      // attention over the cache (positions 0..pos, the new one included)
+      int max_len = 1;
+      for (int r = 0; r < ml; ++r) {
+        int len = a.pos[perm[r]] + 1;
+        if (len > max_len) max_len = len;
+      }
+      int ctas = ml * (dm.Hq / GQ);
+      int want = (592 + ctas - 1) / ctas;
+      if (want < 1) want = 1;
+      if (want > m->lay.max_splits) want = m->lay.max_splits;
+      int split_len = ((max_len + want - 1) / want + 31) / 32 * 32;
+      if (split_len < 32) split_len = 32;
+      int n_splits = (max_len + split_len - 1) / split_len;
+      launches += launch_attention(m->qkv(), m->Kc, m->Vc, m->sched(), l, ml, split_len, n_splits,
+                                   m->lay.max_splits, m->part_o(), m->part_ml(), m->attn_out(), dm, st);
+      // output projection + residual
+      g.W = m->wo[l]; g.R = dm.d; g.K = nq; g.act = m->attn_out(); g.act_stride = nq;
+      g.gain = nullptr; g.out = m->x(); g.out_stride = dm.d;
+      launches += launch_gemv(g, EPI_RESID, ml, st);
+      // RMSNorm + gate/up + SiLU * mul
+      g.W = m->w_gate[l]; g.W2 = m->w_up[l]; g.R = dm.f; g.K = dm.d; g.act = m->x();
+      g.act_stride = dm.d; g.gain = m->mlp_norm[l]; g.out = m->u(); g.out_stride = dm.f;
+      launches += launch_gemv(g, EPI_SWIGLU, ml, st);
+      // down projection + residual
+      g.W = m->w_down[l]; g.W2 = nullptr; g.R = dm.d; g.K = dm.f; g.act = m->u();
+      g.act_stride = dm.f; g.gain = nullptr; g.out = m->x(); g.out_stride = dm.d;
+      launches += launch_gemv(g, EPI_RESID, ml, st);
+    }
+    if (c.kv_fill == D3_FILL_RECOMPUTE && ml < B) {
+      // rows that drop block l: K,V from the block's own norm, W_k, W_v on the carried state
+      g.row_mode = ROWS_SUFFIX;
+      g.W = m->wqkv[l] + (size_t)nq * dm.d; g.W2 = nullptr; g.R = 2 * nkv; g.K = dm.d;
+      g.act = m->x(); g.act_stride = dm.d; g.gain = m->attn_norm[l];
+      g.out = m->qkv(); g.out_stride = dm.qkv_rows; g.out_col0 = nq;
+      launches += launch_gemv(g, EPI_STORE, B - ml, st);
+      launches += launch_rope_append(m->qkv(), m->rope(), m->Kc, m->Vc, m->sched(), l, ROWS_SUFFIX,
+                                     1, B - ml, dm, st);
+      g.out_col0 = 0;
+    }
+  }
+  if (c.kv_fill == D3_FILL_COPY) {
+    bool any = false;
+    for (int b = 0; b < B; ++b) any = any || hi[b] > lo[b];
+    if (any) launches += launch_fill_copy(m->Kc, m->Vc, m->sched(), B, dm, st);
+  }
+  if (logits_dev) {
+    g.layer = 0; g.row_mode = logits_mode;
+    g.W = m->lm_head; g.W2 = nullptr; g.R = dm.V; g.K = dm.d; g.act = m->x(); g.act_stride = dm.d;
+    g.gain = m->final_norm; g.out = logits_dev; g.out_stride = dm.V; g.out_col0 = 0;
+    launches += launch_gemv(g, EPI_LOGITS, logits_mode == ROWS_LAST ? 1 : B, st);
+  }
+  m->last_B = B;
+  for (int b = 0; b < B; ++b) m->last_perm[b] = perm[b];
+  (void)n;
+  if (launches_out) *launches_out = launches;
+  return cudaGetLastError() == cudaSuccess ? D3_OK : D3_ECUDA;
+}
+
+extern "C" {
+
+int32_t d3_depth(int32_t L, double alpha, int64_t i) {
+  if (L < 0 || i < 0 || !alpha_ok(alpha)) return D3_EINVAL;
+  return depth_host(L, alpha, i);
+}
+
+int32_t d3_schedule(int32_t L, double alpha, int32_t start_id, int32_t anchor, int32_t batch,
+                    const int32_t *gen_index, int32_t *n, int32_t *lo, int32_t *hi, int32_t *perm,
+                    int32_t *m_per_layer, int64_t *rows_layers, int32_t *layers_touched) {
+  if (L < 1 || L > D3_MAX_LAYERS || !alpha_ok(alpha) || start_id < 0 || start_id > L ||
+      (anchor != D3_ANCHOR_START && anchor != D3_ANCHOR_TAIL) || batch < 1 ||
+      batch > D3_MAX_BATCH || !gen_index || !n || !lo || !hi || !perm || !m_per_layer)
+    return D3_EINVAL;
+  for (int b = 0; b < batch; ++b)
+    if (gen_index[b] < 0) return D3_EINVAL;
+  for (int b = 0; b < batch; ++b) {
+    int32_t nb = depth_host(L, alpha, gen_index[b]);
+    if (anchor == D3_ANCHOR_TAIL) {
+      lo[b] = nb; hi[b] = L;
+    } else {
+      if (nb < start_id) nb = start_id;
+      lo[b] = start_id; hi[b] = start_id + (L - nb);
+    }
+    n[b] = nb;
+  }
+  // counting sort by n descending, stable in the row index
+  int32_t count[D3_MAX_LAYERS + 2];
+  memset(count, 0, sizeof(count));
+  for (int b = 0; b < batch; ++b) count[L - n[b] + 1]++;
+  for (int k = 1; k <= L + 1; ++k) count[k] += count[k - 1];
+  for (int b = 0; b < batch; ++b) perm[count[L - n[b]]++] = b;
+  int64_t tot = 0;
+  int32_t touched = 0;
+  for (int l = 0; l < L; ++l) {
+    int32_t ml = 0;
+    for (int b = 0; b < batch; ++b) ml += (lo[b] <= l && l < hi[b]) ? 0 : 1;
+    m_per_layer[l] = ml;
+    tot += ml;
+    touched += ml > 0;
+  }
+  if (rows_layers) *rows_layers = tot;
+  if (layers_touched) *layers_touched = touched;
+  return D3_OK;
+}
+
+int32_t d3_workspace_bytes(const d3_config *cfg, size_t *kv_bytes, size_t *scratch_bytes) {
+  if (!config_ok(cfg) || !kv_bytes || !scratch_bytes) return D3_EINVAL;
+  *kv_bytes = 2 * (size_t)cfg->n_layers * cfg->max_slots * cfg->n_kv_heads * cfg->max_seq *
+              cfg->head_dim * sizeof(bf16);
+  *scratch_bytes = make_layout(*cfg).total;
+  return D3_OK;
+}
+
+int32_t d3_load(const d3_config *cfg, const d3_weights *w, void *kv_dev, void *scratch_dev,
+                void *cuda_stream, d3_model **out) {
+  if (!config_ok(cfg) || !w || !kv_dev || !scratch_dev || !out) return D3_EINVAL;
+  if (!w->embed_dev || !w->lm_head_dev || !w->final_norm_dev || !w->attn_norm_dev || !w->wqkv_dev ||
+      !w->wo_dev || !w->mlp_norm_dev || !w->w_gate_dev || !w->w_up_dev || !w->w_down_dev)
+    return D3_EINVAL;
+  auto misaligned = [](const void *p, size_t a) { return p == nullptr || ((uintptr_t)p % a) != 0; };
+  if (misaligned(kv_dev, 256) || misaligned(scratch_dev, 256)) return D3_EINVAL;
+  if (misaligned(w->embed_dev, 16) || misaligned(w->lm_head_dev, 16) || misaligned(w->final_norm_dev, 16))
+    return D3_EINVAL;
+  const int L = cfg->n_layers;
+  for (int l = 0; l < L; ++l)
+    if (misaligned(w->attn_norm_dev[l], 16) || misaligned(w->wqkv_dev[l], 16) ||
+        misaligned(w->wo_dev[l], 16) || misaligned(w->mlp_norm_dev[l], 16) ||
+        misaligned(w->w_gate_dev[l], 16) || misaligned(w->w_up_dev[l], 16) ||
+        misaligned(w->w_down_dev[l], 16))
+      return D3_EINVAL;
+  d3_model *m = new (std::nothrow) d3_model();
+  if (!m) return D3_EINVAL;
+  m->cfg = *cfg;
+  m->dm = Dims{cfg->n_layers, cfg->d_model, cfg->n_q_heads, cfg->n_kv_heads, cfg->head_dim,
+               cfg->d_ffn, cfg->vocab, cfg->max_slots, cfg->max_seq,
+               (cfg->n_q_heads + 2 * cfg->n_kv_heads) * cfg->head_dim};
+  m->lay = make_layout(*cfg);
+  m->stream = (cudaStream_t)cuda_stream;
+  m->embed = (const bf16 *)w->embed_dev;
+  m->lm_head = (const bf16 *)w->lm_head_dev;
+  m->final_norm = (const bf16 *)w->final_norm_dev;
+  for (int l = 0; l < L; ++l) {
+    m->attn_norm.push_back((const bf16 *)w->attn_norm_dev[l]);
+    m->wqkv.push_back((const bf16 *)w->wqkv_dev[l]);
+    m->wo.push_back((const bf16 *)w->wo_dev[l]);
+    m->mlp_norm.push_back((const bf16 *)w->mlp_norm_dev[l]);
+    m->w_gate.push_back((const bf16 *)w->w_gate_dev[l]);
+    m->w_up.push_back((const bf16 *)w->w_up_dev[l]);
+    m->w_down.push_back((const bf16 *)w->w_down_dev[l]);
+  }
+  size_t kv_half = (size_t)L * cfg->max_slots * cfg->n_kv_heads * cfg->max_seq * cfg->head_dim;
+  m->Kc = (bf16 *)kv_dev;
+  m->Vc = m->Kc + kv_half;
+  m->scratch = (char *)scratch_dev;
+  m->pos.assign(cfg->max_slots, -1);
+  m->last_B = 0;
+  const int64_t d = cfg->d_model, f = cfg->d_ffn;
+  m->layer_bytes = 2 * ((int64_t)m->dm.qkv_rows * d + d * cfg->n_q_heads * cfg->head_dim + 3 * d * f + 2 * d);
+  m->head_bytes = 2 * ((int64_t)cfg->vocab * d + d);
+  if (init_kernel_attributes() != 0) { delete m; return D3_ECUDA; }
+  if (cudaMemsetAsync(m->sched(), 0, sizeof(DevSched), m->stream) != cudaSuccess) { delete m; return D3_ECUDA; }
+  launch_rope_table(m->rope(), cfg->max_seq, cfg->head_dim, cfg->rope_base, m->stream);
+  if (cudaGetLastError() != cudaSuccess) { delete m; return D3_ECUDA; }
+  *out = m;
+  return D3_OK;
+}
+
+int32_t d3_prefill(d3_model *m, int32_t slot, const int32_t *tokens, int32_t n_tokens,
+                   float *logits_dev) {
+  if (!m || !tokens || slot < 0 || slot >= m->cfg.max_slots || n_tokens < 1) return D3_EINVAL;
+  if (n_tokens > m->cfg.max_seq) return D3_ECAPACITY;
+  for (int t = 0; t < n_tokens; ++t)
+    if (tokens[t] < 0 || tokens[t] >= m->cfg.vocab) return D3_EINVAL;
+  const int L = m->cfg.n_layers, MB = m->cfg.max_batch;
+  const int32_t *thr = thr_for(m, 1.0);
+  int32_t n[D3_MAX_BATCH], lo[D3_MAX_BATCH], hi[D3_MAX_BATCH], perm[D3_MAX_BATCH], m_l[D3_MAX_LAYERS];
+  for (int t0 = 0; t0 < n_tokens; t0 += MB) {
+    StepArgs a;
+    memset(&a, 0, sizeof(a));
+    a.B = (n_tokens - t0 < MB) ? n_tokens - t0 : MB;
+    a.L = L; a.start_id = m->cfg.start_id; a.anchor = m->cfg.anchor;
+    memcpy(a.thr, thr, sizeof(a.thr));
+    for (int b = 0; b < a.B; ++b) {
+      a.slot[b] = slot; a.tok[b] = tokens[t0 + b]; a.gi[b] = 0; a.pos[b] = t0 + b;
+    }
+    d3_schedule(L, 1.0, m->cfg.start_id, m->cfg.anchor, a.B, a.gi, n, lo, hi, perm, m_l, nullptr, nullptr);
+    const bool last = t0 + a.B >= n_tokens;
+    int32_t rc = run_step(m, a, n, lo, hi, perm, m_l, last ? logits_dev : nullptr, ROWS_LAST, nullptr);
+    if (rc != D3_OK) return rc;
+  }
+  m->pos[slot] = n_tokens;
+  return D3_OK;
+}
+
+int32_t d3_decode_step(d3_model *m, int32_t batch, const int32_t *slots, const int32_t *tokens,
+                       const int32_t *gen_index, double alpha, float *logits_dev,
+                       d3_step_stats *stats, const int32_t *tokens_dev) {
+  if (!m || !slots || !gen_index || !logits_dev || (!tokens && !tokens_dev)) return D3_EINVAL;
+  if (batch < 1 || !alpha_ok(alpha)) return D3_EINVAL;
+  if (batch > m->cfg.max_batch) return D3_ECAPACITY;
+  const d3_config &c = m->cfg;
+  for (int b = 0; b < batch; ++b) {
+    if (slots[b] < 0 || slots[b] >= c.max_slots || gen_index[b] < 1) return D3_EINVAL;
+    if (!tokens_dev && (tokens[b] < 0 || tokens[b] >= c.vocab)) return D3_EINVAL;
+  }
+  for (int b = 0; b < batch; ++b) {
+    for (int a2 = 0; a2 < b; ++a2)
+      if (slots[a2] == slots[b]) return D3_ESTATE;
+    if (m->pos[slots[b]] < 1) return D3_ESTATE;
+  }
+  for (int b = 0; b < batch; ++b)
+    if (m->pos[slots[b]] >= c.max_seq) return D3_ECAPACITY;
+
+  const int L = c.n_layers;
+  StepArgs a;
+  memset(&a, 0, sizeof(a));
+  a.B = batch; a.L = L; a.start_id = c.start_id; a.anchor = c.anchor; a.tok_dev = tokens_dev;
+  memcpy(a.thr, thr_for(m, alpha), sizeof(a.thr));
+  for (int b = 0; b < batch; ++b) {
+    a.slot[b] = slots[b]; a.tok[b] = tokens_dev ? 0 : tokens[b]; a.gi[b] = gen_index[b];
+    a.pos[b] = m->pos[slots[b]];
+  }
+  int32_t n[D3_MAX_BATCH], lo[D3_MAX_BATCH], hi[D3_MAX_BATCH], perm[D3_MAX_BATCH], m_l[D3_MAX_LAYERS];
+  int64_t rows_layers = 0;
+  int32_t touched = 0;
+  int32_t rc = d3_schedule(L, alpha, c.start_id, c.anchor, batch, gen_index, n, lo, hi, perm, m_l,
+                           &rows_layers, &touched);
+  if (rc != D3_OK) return rc;
+  int32_t launches = 0;
+  rc = run_step(m, a, n, lo, hi, perm, m_l, logits_dev, ROWS_ALL, &launches);
+  if (rc != D3_OK) return rc;
+  if (stats) {
+    if (stats->n) memcpy(stats->n, n, sizeof(int32_t) * batch);
+    if (stats->m_per_layer) memcpy(stats->m_per_layer, m_l, sizeof(int32_t) * L);
+    stats->rows_layers = rows_layers;
+    stats->layers_touched = touched;
+    stats->kernel_launches = launches;
+    const int64_t kv_tok = 2LL * c.n_kv_heads * c.head_dim * 2;  // K and V of one token, one block
+    int64_t bytes = (int64_t)touched * m->layer_bytes + m->head_bytes;
+    for (int b = 0; b < batch; ++b) {
+      bytes += (int64_t)n[b] * kv_tok * (a.pos[b] + 1);           // KV read by retained blocks
+      int64_t written = n[b] + (c.kv_fill != D3_FILL_NONE ? (hi[b] - lo[b]) : 0);
+      bytes += written * kv_tok;                                   // KV appended / filled
+    }
+    bytes += (int64_t)batch * c.d_model * 2 + (int64_t)batch * c.vocab * 4;
+    stats->algorithmic_bytes = bytes;
+  }
+  for (int b = 0; b < batch; ++b) m->pos[slots[b]] += 1;
+  return D3_OK;
+}
+
+int32_t d3_argmax(d3_model *m, const float *logits_dev, int32_t batch, int32_t *tokens_dev) {
+  if (!m || !logits_dev || !tokens_dev || batch < 1) return D3_EINVAL;
+  launch_argmax(logits_dev, batch, m->cfg.vocab, tokens_dev, m->stream);
+  return cudaGetLastError() == cudaSuccess ? D3_OK : D3_ECUDA;
+}
+
+int32_t d3_read_schedule(d3_model *m, int32_t *n, int32_t *perm, int32_t *m_per_layer,
+                         int64_t *counters) {
+  if (!m) return D3_EINVAL;
+  DevSched h;
+  if (cudaStreamSynchronize(m->stream) != cudaSuccess) return D3_ECUDA;
+  if (cudaMemcpy(&h, m->sched(), sizeof(h), cudaMemcpyDeviceToHost) != cudaSuccess) return D3_ECUDA;
+  if (n) memcpy(n, h.n, sizeof(int32_t) * h.B);
+  if (perm) memcpy(perm, h.perm, sizeof(int32_t) * h.B);
+  if (m_per_layer) memcpy(m_per_layer, h.m, sizeof(int32_t) * h.L);
+  if (counters) { counters[0] = h.rows_layers; counters[1] = h.layers_touched; }
+  return D3_OK;
+}
+
+int32_t d3_read_hidden(d3_model *m, float *hidden) {
+  if (!m || !hidden || m->last_B < 1) return D3_EINVAL;
+  if (cudaStreamSynchronize(m->stream) != cudaSuccess) return D3_ECUDA;
+  const size_t row = (size_t)m->cfg.d_model * 4;
+  for (int r = 0; r < m->last_B; ++r)
+    if (cudaMemcpy((char *)hidden + (size_t)m->last_perm[r] * row, (char *)m->x() + r * row, row,
+                   cudaMemcpyDeviceToHost) != cudaSuccess)
+      return D3_ECUDA;
+  return D3_OK;
+}
+
+int32_t d3_read_kv(d3_model *m, int32_t layer, int32_t slot, int32_t pos, float *k, float *v) {
+  if (!m || !k || !v || layer < 0 || layer >= m->cfg.n_layers || slot < 0 ||
+      slot >= m->cfg.max_slots || pos < 0 || pos >= m->cfg.max_seq)
+    return D3_EINVAL;
+  if (cudaStreamSynchronize(m->stream) != cudaSuccess) return D3_ECUDA;
+  const int dh = m->cfg.head_dim;
+  std::vector<uint16_t> buf(dh);
+  for (int h = 0; h < m->cfg.n_kv_heads; ++h) {
+    size_t off = ((((size_t)layer * m->cfg.max_slots + slot) * m->cfg.n_kv_heads + h) * m->cfg.max_seq + pos) * dh;
+    for (int which = 0; which < 2; ++which) {
+      const bf16 *src = (which ? m->Vc : m->Kc) + off;
+      if (cudaMemcpy(buf.data(), src, dh * 2, cudaMemcpyDeviceToHost) != cudaSuccess) return D3_ECUDA;
+      float *dst = (which ? v : k) + h * dh;
+      for (int e = 0; e < dh; ++e) {
+        uint32_t u = (uint32_t)buf[e] << 16;
+        memcpy(dst + e, &u, 4);
+      }
+    }
+  }
+  return D3_OK;
+}
+
+int32_t d3_slot_pos(const d3_model *m, int32_t slot) {
+  if (!m || slot < 0 || slot >= m->cfg.max_slots) return D3_EINVAL;
+  return m->pos[slot] < 0 ? D3_ESTATE : m->pos[slot];
+}
+
+int32_t d3_reset_slot(d3_model *m, int32_t slot) {
+  if (!m || slot < 0 || slot >= m->cfg.max_slots) return D3_EINVAL;
+  m->pos[slot] = -1;
+  return D3_OK;
+}
+
+int32_t d3_sync(d3_model *m) {
+  if (!m) return D3_EINVAL;
+  if (cudaStreamSynchronize(m->stream) != cudaSuccess) return D3_ECUDA;
+  int32_t status = 0;
+  if (cudaMemcpy(&status, &m->sched()->status, 4, cudaMemcpyDeviceToHost) != cudaSuccess)
+    return D3_ECUDA;
+  return status;
+}
+
+void d3_free(d3_model *m) { delete m; }
+
+const char *d3_strerror(int32_t code) {
+  switch (code) {
+    case D3_OK: return "ok";
+    case D3_EINVAL: return "invalid argument";
+    case D3_ECAPACITY: return "capacity exceeded (max_seq or max_batch)";
+    case D3_ESTATE: return "slot not prefilled, or used twice in one batch";
+    case D3_ECUDA: return "CUDA runtime error";
+    case D3_ETIMEOUT: return "a bounded device-side wait ran out";
+    default: return "unknown error";
+  }
+}
+
+}  // extern "C"

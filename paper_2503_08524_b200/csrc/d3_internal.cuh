@@ -1,0 +1,98 @@
+// Internal declarations shared by the kernels and the C ABI of libd3.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "d3.h"
+
+namespace d3 {
+
+typedef __nv_bfloat16 bf16;
+
+// One step's caller arguments, passed to the schedule kernel by value (kernel
+// parameters are copied at launch, so the host arrays may be reused at once).
+struct StepArgs {
+  int32_t B, L, start_id, anchor;
+  int32_t slot[D3_MAX_BATCH];
+  int32_t tok[D3_MAX_BATCH];
+  int32_t gi[D3_MAX_BATCH];   // generation index i of the row (0 = full depth)
+  int32_t pos[D3_MAX_BATCH];  // cache position the row's token is written to
+  // thr[n] = smallest i with floor(L alpha^i) < n, for n = 1..L (thr[0] unused)
+  int32_t thr[D3_MAX_LAYERS + 1];
+  const int32_t *tok_dev;     // nullable: device token ids that replace tok[]
+};
+
+// The schedule of the running step in device memory (written by the schedule
+// kernel, read by every other kernel).  "_s" arrays are in sorted row order.
+struct DevSched {
+  int32_t B, L;
+  int32_t n[D3_MAX_BATCH];     // caller order
+  int32_t perm[D3_MAX_BATCH];  // sorted index -> caller row
+  int32_t slot_s[D3_MAX_BATCH], pos_s[D3_MAX_BATCH], tok_s[D3_MAX_BATCH];
+  int32_t lo_s[D3_MAX_BATCH], hi_s[D3_MAX_BATCH];
+  int32_t m[D3_MAX_LAYERS];    // rows that run block l = a prefix of the sorted order
+  long long rows_layers;
+  int32_t layers_touched;
+  int32_t status;              // 0, or a D3_E* code detected on the device
+};
+
+// Which rows of the sorted batch a kernel works on.
+enum RowMode {
+  ROWS_PREFIX = 0,  // [0, m[layer])        rows that run the block
+  ROWS_SUFFIX = 1,  // [m[layer], B)        rows that drop it (recompute fill)
+  ROWS_ALL = 2,     // [0, B)
+  ROWS_LAST = 3     // [B-1, B)             prefill: only the last position needs logits
+};
+
+enum Epilogue {
+  EPI_STORE = 0,   // out[row][r] = y
+  EPI_RESID = 1,   // out[row][r] += y          (residual stream)
+  EPI_SWIGLU = 2,  // out[row][r] = silu(W y) * (W2 y)
+  EPI_LOGITS = 3   // out[caller row][r] = y    (un-permuted)
+};
+
+struct GemvArgs {
+  const bf16 *W, *W2;   // [R][K] row-major (W2: second matrix of EPI_SWIGLU)
+  int R, K;
+  const float *act;     // [rows][act_stride]
+  int act_stride;
+  const bf16 *gain;     // nullable: RMSNorm gain fused on the activation
+  float eps;
+  float *out;
+  int out_stride;
+  int out_col0;         // column offset added to the output row index r
+  const DevSched *sched;
+  int layer;
+  int row_mode;
+};
+
+struct Dims {
+  int L, d, Hq, Hkv, dh, f, V, max_slots, max_seq, qkv_rows;
+};
+
+// Byte offsets of the regions of the caller's scratch buffer.
+struct Layout {
+  size_t sched, rope, x, qkv, attn_out, part_o, part_ml, u, total;
+  int max_splits;
+};
+
+Layout make_layout(const d3_config &c);
+
+// launchers (each enqueues on `st`; returns the number of kernels launched)
+int launch_rope_table(float2 *table, int max_seq, int dh, float base, cudaStream_t st);
+int launch_schedule_embed(const StepArgs &a, DevSched *s, const bf16 *E, float *x, int d,
+                          cudaStream_t st);
+int launch_gemv(const GemvArgs &g, int epi, int m_rows, cudaStream_t st);
+int launch_rope_append(float *qkv, const float2 *rope, bf16 *Kc, bf16 *Vc, const DevSched *s,
+                       int layer, int row_mode, int kv_only, int m_rows, const Dims &dm,
+                       cudaStream_t st);
+int launch_attention(const float *qkv, const bf16 *Kc, const bf16 *Vc, const DevSched *s, int layer,
+                     int m_rows, int split_len, int n_splits, int max_splits, float *part_o,
+                     float *part_ml, float *attn_out, const Dims &dm, cudaStream_t st);
+int launch_fill_copy(bf16 *Kc, bf16 *Vc, const DevSched *s, int B, const Dims &dm, cudaStream_t st);
+int launch_argmax(const float *logits, int B, int V, int32_t *out, cudaStream_t st);
+int init_kernel_attributes();
+
+}  // namespace d3
