@@ -162,7 +162,7 @@ class D3Model:
         self.h = h
 
     def close(self):
-        if getattr(self, "h", None):
+        if getattr(self, "h", None) and LIB is not None:
             LIB.d3_free(self.h)
             self.h = None
 

@@ -401,6 +401,9 @@ k_attn_partial(const float *qkv, const bf16 *Kc, const bf16 *Vc, const DevSched 
   const int slot = s->slot_s[row];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, part = lane & 7;
   const int worker = warp * 4 + (lane >> 3);
+  // the 8 lanes of a worker run the position loop in lockstep; other workers of
+  // the warp may run fewer iterations, so in-loop shuffles name only the worker
+  const unsigned wmask = 0xffu << (lane & 24);
 
   float q[GQ][EPL];
   const float scale = rsqrtf((float)DH);
@@ -443,9 +446,9 @@ k_attn_partial(const float *qkv, const bf16 *Kc, const bf16 *Vc, const DevSched 
       float sc = 0.f;
 #pragma unroll
       for (int e = 0; e < EPL; ++e) sc += q[g][e] * kf[e];
-      sc += __shfl_xor_sync(0xffffffffu, sc, 1);
-      sc += __shfl_xor_sync(0xffffffffu, sc, 2);
-      sc += __shfl_xor_sync(0xffffffffu, sc, 4);
+      sc += __shfl_xor_sync(wmask, sc, 1);
+      sc += __shfl_xor_sync(wmask, sc, 2);
+      sc += __shfl_xor_sync(wmask, sc, 4);
       float mn = fmaxf(mx[g], sc);
       float corr = __expf(mx[g] - mn), p = __expf(sc - mn);
       mx[g] = mn;

@@ -1,0 +1,270 @@
+"""Parity of the CUDA path with the CPU oracle, through the C ABI (GPU)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle as O
+from paper_2503_08524_b200 import inputs as I
+
+from parity import LOGITS_MAX_ABS, check_step, make_pair, rel_l2
+
+pytestmark = pytest.mark.gpu
+SEED = I.BASE_SEED
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2503_08524_b200 import binding
+    assert torch.cuda.is_available()
+    return binding
+
+
+# ------------------------------------------------------------ depth schedule (K0)
+
+@pytest.mark.parametrize("anchor", [0, 1])
+def test_schedule_kernel_is_bit_exact(B, anchor):
+    shape = I.TINY
+    rng = np.random.default_rng(3)
+    for start, alpha in [(0, 0.95), (1, 0.98), (2, 0.9), (0, 1.0), (4, 0.5)]:
+        orc, gpu = make_pair(shape, SEED, 64, 8, 64, start_id=start, anchor=anchor, kv_fill=0)
+        for s in range(64):
+            gpu.d3_prefill(s, [1, 2])
+        for Bn in (1, 2, 3, 17, 64):
+            gi = rng.integers(1, 60, size=Bn).astype(np.int32)
+            gi[Bn // 2] = gi[0]
+            slots = rng.permutation(64)[:Bn]
+            _, st = gpu.d3_decode_step(slots, [5] * Bn, gi, alpha, want_stats=True)
+            dev = gpu.d3_read_schedule(Bn)
+            want = O.schedule(shape.n_layers, alpha, start, anchor, gi)
+            host = B.d3_schedule(shape.n_layers, alpha, start, anchor, gi)
+            for k in ("n", "perm", "m_per_layer"):
+                assert np.array_equal(dev[k], want[k]), (k, Bn, start, alpha)
+                assert np.array_equal(host[k], want[k])
+            assert np.array_equal(st["n"], want["n"]) and np.array_equal(st["m_per_layer"], want["m_per_layer"])
+            for k in ("rows_layers", "layers_touched"):
+                assert dev[k] == want[k] == st[k]
+            for s in slots:
+                gpu.d3_reset_slot(int(s))
+                gpu.d3_prefill(int(s), [1, 2])
+        gpu.close()
+
+
+def test_schedule_kernel_large_L(B):
+    # 7B/13B/70B layer counts on a narrow model: only the integers matter here
+    for L, alpha, start in [(32, 0.997, 6), (40, 0.998, 8), (80, 0.998, 16), (128, 0.99, 25)]:
+        shape = I.ModelShape("narrow", L, 64, 2, 1, 32, 64, 128)
+        orc, gpu = make_pair(shape, SEED, 32, 4, 32, start_id=start, kv_fill=1)
+        for s in range(32):
+            gpu.d3_prefill(s, [3])
+        gi = np.array([1 + (8 * b) % 256 for b in range(32)], np.int32)
+        gpu.d3_decode_step(list(range(32)), [7] * 32, gi, alpha)
+        dev = gpu.d3_read_schedule(32)
+        want = O.schedule(L, alpha, start, 0, gi)
+        for k in ("n", "perm", "m_per_layer"):
+            assert np.array_equal(dev[k], want[k]), (k, L)
+        assert dev["rows_layers"] == want["rows_layers"] and dev["layers_touched"] == want["layers_touched"]
+        gpu.close()
+
+
+# --------------------------------------------------- tiny config, batch 1, whole run
+
+@pytest.mark.parametrize("shape", [I.TINY, I.TINY_GQA], ids=["mha", "gqa"])
+@pytest.mark.parametrize("alpha", [1.0, 0.98, 0.95])
+@pytest.mark.parametrize("kv_round", [False, True], ids=["kv-exact", "kv-bf16"])
+def test_tiny_generate_teacher_forced(B, shape, alpha, kv_round):
+    orc, gpu = make_pair(shape, SEED, 2, 64, 1, start_id=0, kv_round_bf16=kv_round)
+    prompt = I.prompt_tokens(shape, SEED, 0, 16).numpy()
+    o_lg, o_hid = orc.prefill(1, prompt, want_hidden=True)
+    g_lg = gpu.d3_prefill(1, prompt)
+    check_step("prefill", g_lg.cpu().numpy()[None], gpu.d3_read_hidden(1)[-1:], o_lg[None], o_hid[None])
+    tok = O.argmax(o_lg)
+    layers = 0
+    for i in range(1, 32):
+        r = orc.decode_step([1], [tok], [i], alpha)
+        g, st = gpu.d3_decode_step([1], [tok], [i], alpha, want_stats=True)
+        check_step(f"step {i}", g.cpu().numpy(), gpu.d3_read_hidden(1), r["logits"], r["hidden"])
+        assert st["n"][0] == O.window(shape.n_layers, alpha, i, 0)[0]
+        layers += st["rows_layers"]
+        tok = O.argmax(r["logits"][0])
+    assert layers == sum(O.depth(shape.n_layers, alpha, i) for i in range(1, 32))
+    assert gpu.d3_slot_pos(1) == orc.slot_pos(1) == 16 + 31
+    gpu.close()
+
+
+def test_tiny_greedy_tokens_identical(B):
+    # free-running greedy decode, argmax on the device, fed back on the device
+    shape = I.TINY
+    for alpha in (1.0, 0.98, 0.95):
+        orc, gpu = make_pair(shape, SEED + 1, 1, 64, 1, gain_jitter=0.0, kv_round_bf16=False)
+        prompt = I.prompt_tokens(shape, SEED + 1, 0, 16).numpy()
+        o_tok = [O.argmax(orc.prefill(0, prompt))]
+        margins = []
+        for i in range(1, 32):
+            lg = orc.decode_step([0], [o_tok[-1]], [i], alpha)["logits"][0]
+            top = np.sort(lg)[-2:]
+            margins.append(top[1] - top[0])
+            o_tok.append(O.argmax(lg))
+        lg = gpu.d3_prefill(0, prompt)
+        tok = gpu.d3_argmax(lg)
+        g_tok = [int(tok.item())]
+        for i in range(1, 32):
+            lg = gpu.d3_decode_step([0], None, [i], alpha, tokens_dev=tok)
+            tok = gpu.d3_argmax(lg)
+            g_tok.append(int(tok.item()))
+        if min(margins) > 4 * LOGITS_MAX_ABS:
+            assert g_tok == o_tok, alpha
+        else:   # a near-tie may legitimately flip: compare up to the first such step
+            k = next(j for j, m in enumerate(margins) if m <= 4 * LOGITS_MAX_ABS) + 1
+            assert g_tok[:k] == o_tok[:k], alpha
+        gpu.close()
+
+
+# ------------------------------------------------ mixed-depth batches, anchors, fills
+
+@pytest.mark.parametrize("anchor,start", [(0, 0), (0, 1), (0, 2), (1, 0)])
+@pytest.mark.parametrize("fill", [0, 1, 2])
+def test_batched_mixed_depth_steps(B, anchor, start, fill):
+    shape = I.TINY_GQA
+    Bn, alpha = 7, 0.96
+    orc, gpu = make_pair(shape, SEED + 2, 8, 96, 8, start_id=start, anchor=anchor, kv_fill=fill)
+    gpu.poison_kv()
+    orc.poison_kv()
+    lens = I.uniform_ints(SEED + 2, 77, Bn, 3, 40)
+    slots = [5, 0, 7, 2, 3, 6, 1]
+    for b in range(Bn):
+        p = I.prompt_tokens(shape, SEED + 2, b, lens[b]).numpy()
+        o = orc.prefill(slots[b], p)
+        g = gpu.d3_prefill(slots[b], p)
+        check_step(f"prefill {b}", g.cpu().numpy()[None], None, o[None], None)
+    gi0 = [1, 9, 30, 2, 55, 17, 9]
+    seen = set()
+    for step in range(12):
+        toks = I.token_ids(SEED + 2, 500 + step, Bn, shape.vocab).numpy()
+        gi = [g + step for g in gi0]
+        r = orc.decode_step(slots, toks, gi, alpha)
+        g, st = gpu.d3_decode_step(slots, toks, gi, alpha, want_stats=True)
+        check_step(f"step {step}", g.cpu().numpy(), gpu.d3_read_hidden(Bn), r["logits"], r["hidden"])
+        seen.update(int(v) for v in st["n"])
+    assert len(seen) >= 2
+    # the caches agree wherever the oracle holds a number (bf16 storage on the GPU)
+    for b in range(Bn):
+        pos = orc.slot_pos(slots[b]) - 1
+        for l in range(shape.n_layers):
+            ok, ov = orc.read_kv(l, slots[b], pos)
+            gk, gv = gpu.d3_read_kv(l, slots[b], pos)
+            if np.isnan(ok).any():
+                assert np.isnan(gk).all() and np.isnan(gv).all()      # FILL_NONE leaves it alone
+            else:
+                assert np.abs(gk - ok).max() <= 0.02 * max(1.0, np.abs(ok).max())
+                assert np.abs(gv - ov).max() <= 0.02 * max(1.0, np.abs(ov).max())
+    gpu.close()
+
+
+@pytest.mark.parametrize("fill", [1, 2])
+def test_alpha_raised_mid_sequence_reads_filled_entries(B, fill):
+    # depth grows again when the caller raises alpha: later tokens then read what
+    # the fill mode left in the cache (defined by the fill rule only)
+    shape = I.TINY
+    orc, gpu = make_pair(shape, SEED + 3, 1, 64, 1, start_id=1, kv_fill=fill)
+    prompt = I.prompt_tokens(shape, SEED + 3, 0, 8).numpy()
+    tok = O.argmax(orc.prefill(0, prompt))
+    gpu.d3_prefill(0, prompt)
+    for i in range(1, 24):
+        alpha = 0.9 if i < 12 else 1.0
+        r = orc.decode_step([0], [tok], [i], alpha)
+        g = gpu.d3_decode_step([0], [tok], [i], alpha)
+        check_step(f"step {i}", g.cpu().numpy(), gpu.d3_read_hidden(1), r["logits"], r["hidden"])
+        tok = O.argmax(r["logits"][0])
+    gpu.close()
+
+
+def test_prefill_longer_than_a_batch_and_ragged_lengths(B):
+    shape = I.TINY
+    orc, gpu = make_pair(shape, SEED + 4, 3, 200, 16)
+    for slot, n in [(0, 1), (1, 16), (2, 17), (0, 131)]:
+        p = I.prompt_tokens(shape, SEED + 4, slot + n, n).numpy()
+        o, oh = orc.prefill(slot, p, want_hidden=True)
+        g = gpu.d3_prefill(slot, p)
+        check_step(f"prefill {n}", g.cpu().numpy()[None], None, o[None], None)
+        assert gpu.d3_slot_pos(slot) == n
+    # long context decode: several attention splits with a ragged tail
+    tok = 3
+    for i in range(1, 6):
+        r = orc.decode_step([0, 2], [tok, tok], [i, i + 3], 0.97)
+        g = gpu.d3_decode_step([0, 2], [tok, tok], [i, i + 3], 0.97)
+        check_step(f"step {i}", g.cpu().numpy(), gpu.d3_read_hidden(2), r["logits"], r["hidden"])
+    gpu.close()
+
+
+# ----------------------------------------------------------- production widths
+
+@pytest.mark.parametrize("base,layers,Bn", [(I.LLAMA_7B, 3, 1), (I.LLAMA_7B, 2, 5), (I.LLAMA_70B, 2, 3)],
+                         ids=["7b-width-b1", "7b-width-b5", "70b-width-gqa-b3"])
+def test_production_widths(B, base, layers, Bn):
+    # full-width blocks (same kernel shapes and tiling as the benchmark), few layers
+    shape = base.with_layers(layers)
+    orc, gpu = make_pair(shape, SEED + 5, Bn, 96, 8, start_id=1, gain_jitter=0.1)
+    lens = I.uniform_ints(SEED + 5, 3, Bn, 5, 40)
+    for b in range(Bn):
+        p = I.prompt_tokens(shape, SEED + 5, b, lens[b]).numpy()
+        o = orc.prefill(b, p)
+        g = gpu.d3_prefill(b, p)
+        check_step(f"prefill {b}", g.cpu().numpy()[None], None, o[None], None)
+    for step in range(3):
+        toks = I.token_ids(SEED + 5, 40 + step, Bn, shape.vocab).numpy()
+        gi = [1 + step + 2 * b for b in range(Bn)]
+        alpha = 0.8
+        r = orc.decode_step(list(range(Bn)), toks, gi, alpha)
+        g = gpu.d3_decode_step(list(range(Bn)), toks, gi, alpha)
+        check_step(f"step {step}", g.cpu().numpy(), gpu.d3_read_hidden(Bn), r["logits"], r["hidden"])
+    gpu.close()
+
+
+# ------------------------------------------------------------------ error paths
+
+def test_error_paths_change_no_state(B):
+    shape = I.TINY
+    orc, gpu = make_pair(shape, SEED, 2, 8, 2)
+    lg = torch.empty((2, shape.vocab), dtype=torch.float32, device="cuda:0")
+
+    def code(**kw):
+        args = dict(slots=[0], tokens=[1], gen_index=[1], alpha=0.9)
+        args.update(kw)
+        with pytest.raises(B.D3Error) as e:
+            gpu.d3_decode_step(**args)
+        return e.value.code
+
+    assert code() == B.ESTATE                                   # never prefilled
+    gpu.d3_prefill(0, [1, 2, 3])
+    gpu.d3_prefill(1, [1, 2, 3])
+    assert code(slots=[0, 0], tokens=[1, 1], gen_index=[1, 1]) == B.ESTATE
+    assert code(gen_index=[0]) == B.EINVAL
+    assert code(tokens=[shape.vocab]) == B.EINVAL
+    assert code(slots=[2]) == B.EINVAL
+    assert code(alpha=0.0) == B.EINVAL and code(alpha=float("nan")) == B.EINVAL
+    assert code(slots=[0, 1, 0], tokens=[1] * 3, gen_index=[1] * 3) == B.ECAPACITY   # > max_batch
+    assert gpu.d3_slot_pos(0) == 3 and gpu.d3_slot_pos(1) == 3
+    for i in range(5):
+        gpu.d3_decode_step([0], [1], [i + 1], 0.9)
+    assert code(gen_index=[6]) == B.ECAPACITY                   # cache full
+    with pytest.raises(B.D3Error) as e:
+        gpu.d3_prefill(1, list(range(9)))
+    assert e.value.code == B.ECAPACITY
+    gpu.d3_sync()
+    gpu.d3_reset_slot(0)
+    assert gpu.d3_slot_pos(0) == B.ESTATE
+    gpu.close()
+
+
+def test_argmax_lowest_index_on_ties(B):
+    shape = I.TINY
+    orc, gpu = make_pair(shape, SEED, 1, 8, 4)
+    lg = torch.zeros((4, shape.vocab), dtype=torch.float32, device="cuda:0")
+    lg[0, 100] = 3.0
+    lg[0, 900] = 3.0
+    lg[1, 1023] = 1.0
+    lg[2] = -5.0
+    lg[3, 0] = 9.0
+    out = gpu.d3_argmax(lg).cpu().tolist()
+    assert out == [100, 1023, 0, 0]
+    gpu.close()
