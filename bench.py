@@ -1,0 +1,389 @@
+#!/usr/bin/env python
+"""Benchmark of the D3 decode hot path on B200.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--alpha A] [--impl d3|reference]
+
+One "step" is one decode step of the whole hot path (schedule, every retained
+block, KV fill, final norm + LM head) for the batch.  The workload is the
+Llama-2-7B-shaped decoder (random-init bf16, seeded), batch 1, prompt 512
+uniform-random token ids, generate 256; the K timed steps take their generation
+indices i evenly over 1..255 (K = 255, the default, is the run itself).
+
+Prints ONE JSON line: decode tokens/s (device-timed, inputs resident in HBM),
+the HBM roofline of the dominant kernel and of the whole step, the same metric
+end to end through the C ABI with host buffers, the alpha = 1 run of the same
+kernels, and the CPU oracle timed on the host cores as a baseline.
+`--impl reference` times the CPU oracle alone on a bounded sample.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+from paper_2503_08524_b200 import inputs as I
+
+PROMPT, GENERATE, BATCH = 512, 256, 1
+START_FRACTION = 0.2          # the paper's GSM8K value of `start`
+METRIC = "decode tokens/s at 1 B200 and % of HBM roofline (retained-layer bytes/step)"
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+ORACLE_PROMPT = 32            # bounded sample for the CPU oracle
+
+
+def gen_indices(k: int):
+    """Generation index of each of k steps, spread evenly over the run 1..GENERATE-1."""
+    n = GENERATE - 1
+    if k >= n:
+        return [1 + (j % n) for j in range(k)]
+    return [1 + (j * n) // k for j in range(k)]
+
+
+def measured_peak():
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle-reason samples taken while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, device_index: int):
+        self.tmp = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        sel = str(device_index)
+        try:
+            sel = "GPU-" + str(torch.cuda.get_device_properties(device_index).uuid)
+        except Exception:
+            pass
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", sel, "--query-gpu=" + self.FIELDS,
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=self.tmp, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.tmp.flush()
+        self.tmp.seek(0)
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.tmp.read().splitlines():
+            p = [v.strip() for v in line.split(",")]
+            if len(p) < 7:
+                continue
+            try:
+                sm.append(float(p[0]))
+                mx.append(float(p[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, p[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        self.tmp.close()
+        os.unlink(self.tmp.name)
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons),
+                       samples=len(sm))
+        return out
+
+
+def time_oracle(shape, w_cpu, alpha, start_id, steps, warmup):
+    """CPU oracle on a bounded sample: ORACLE_PROMPT-token prefill (untimed), then
+    `steps` timed decode steps with the same generation indices as the GPU run."""
+    import oracle as O
+    orc = O.Oracle(shape, w_cpu, 1, ORACLE_PROMPT + steps + warmup + 2, start_id=start_id)
+    prompt = I.prompt_tokens(shape, I.BASE_SEED, 0, ORACLE_PROMPT).numpy()
+    orc.prefill(0, prompt)
+    toks = I.token_ids(I.BASE_SEED, 999, steps + warmup, shape.vocab).numpy()
+    gi = gen_indices(steps)
+    for j in range(warmup):
+        orc.decode_step([0], [int(toks[j])], [gi[0]], alpha)
+    t0 = time.perf_counter()
+    for j in range(steps):
+        orc.decode_step([0], [int(toks[warmup + j])], [gi[j]], alpha)
+    dt = time.perf_counter() - t0
+    orc.close()
+    return steps * BATCH / dt, dt, O.threads()
+
+
+def host_mem_available_gb():
+    try:
+        for line in open("/proc/meminfo"):
+            if line.startswith("MemAvailable"):
+                return int(line.split()[1]) / 1e6
+    except Exception:
+        pass
+    return 0.0
+
+
+def oracle_shape_and_scale(shape):
+    """The full 32-block model if host RAM holds its bf16 weights, else 8 blocks
+    (the result is then scaled by the block count and says so)."""
+    need_gb = (shape.n_layers * shape.layer_weight_bytes + 2 * shape.head_weight_bytes) / 1e9
+    if host_mem_available_gb() > need_gb + 16:
+        return shape, 1.0, f"{shape.n_layers} blocks"
+    small = shape.with_layers(8)
+    return small, 8.0 / shape.n_layers, "8 of 32 blocks, tokens/s scaled by 8/32"
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    shape, scale, note = oracle_shape_and_scale(I.LLAMA_7B)
+    dev = "cuda:0" if torch.cuda.is_available() else "cpu"
+    w = I.make_weights(shape, I.BASE_SEED, device=dev)
+    w_cpu = I.weights_to(w, "cpu")
+    del w
+    start_id = int(START_FRACTION * I.LLAMA_7B.n_layers)
+    steps = min(args.steps, 64)
+    tps, dt, cores = time_oracle(shape, w_cpu, args.alpha, min(start_id, shape.n_layers), steps,
+                                 min(args.warmup, 3))
+    tps *= scale
+    sample = (f"CPU oracle (fp64, OpenMP), 7B shape, {note}, prompt {ORACLE_PROMPT}, "
+              f"{steps} decode steps at alpha={args.alpha}")
+    line = {
+        "impl": "reference", "metric": METRIC, "value": tps, "unit": "tokens/s",
+        "n_gpus": args.gpus, "steps": steps, "warmup": min(args.warmup, 3),
+        "ms_per_step": 1e3 * dt / steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": "llama2-7b-shape batch 1, prompt 512, generate 256 (oracle: bounded sample)",
+                   "alpha": args.alpha, "start_id": start_id},
+        "cpu_baseline": {"value": tps, "unit": "tokens/s", "cores": cores, "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": tps, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=GENERATE - 1)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--alpha", type=float, default=0.995)
+    ap.add_argument("--impl", default="d3", choices=["d3", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--layers", type=int, default=0,
+                    help="profiling aid: keep only this many blocks (same kernel shapes, less memory); "
+                         "numbers from such a run are not benchmark values")
+    ap.add_argument("--prompt", type=int, default=PROMPT, help="profiling aid: shorter prompt")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+    if args.impl == "reference":
+        return run_reference(args)
+
+    from paper_2503_08524_b200 import binding as B   # raises if libd3 is missing
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (no CPU fallback)")
+    torch.cuda.set_device(local)
+    dev = f"cuda:{local}"
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device(dev))
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    shape = I.LLAMA_7B if args.layers <= 0 else I.LLAMA_7B.with_layers(args.layers)
+    start_id = int(START_FRACTION * shape.n_layers)
+    K, W = args.steps, args.warmup
+    max_seq = args.prompt + K + W + 8
+    w = I.make_weights(shape, I.BASE_SEED, device=dev)
+    # max_batch 32 only lets the (untimed) prefill run 32 prompt positions per pass
+    model = B.D3Model(shape, w, 1, max_seq, 32, start_id=start_id, device=dev)
+    model.zero_kv()
+    prompt = I.prompt_tokens(shape, I.BASE_SEED, 0, args.prompt).numpy()
+    toks = I.token_ids(I.BASE_SEED, 999, K + W, shape.vocab).numpy()
+    gi = gen_indices(K)
+    logits = torch.empty((BATCH, shape.vocab), dtype=torch.float32, device=dev)
+    stream = torch.cuda.current_stream()
+
+    def timed_run(alpha, profile=False):
+        """Prefill, W warm-up steps, K timed steps.  Returns (ms, stats totals)."""
+        model.d3_reset_slot(0)
+        model.d3_prefill(0, prompt)
+        for j in range(W):
+            model.d3_decode_step([0], [int(toks[j])], [gi[0]], alpha, logits=logits)
+        model.d3_profile(profile)
+        if profile:
+            model.d3_read_profile()
+        tot = {"bytes": 0, "rows_layers": 0, "launches": 0, "touched": 0}
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        e0.record(stream)
+        for j in range(K):
+            _, st = model.d3_decode_step([0], [int(toks[W + j])], [gi[j]], alpha, logits=logits,
+                                         want_stats=True)
+            tot["bytes"] += st["algorithmic_bytes"]
+            tot["rows_layers"] += st["rows_layers"]
+            tot["launches"] += st["kernel_launches"]
+            tot["touched"] += st["layers_touched"]
+        e1.record(stream)
+        barrier()
+        ms = e0.elapsed_time(e1)
+        prof = model.d3_read_profile() if profile else None
+        model.d3_profile(False)
+        return ms, tot, prof
+
+    def max_over_ranks(ms):
+        if dist is None:
+            return ms
+        t = torch.tensor([ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    # ---- main timed region (clock samples taken meanwhile)
+    sampler = ClockSampler(local) if rank == 0 else None
+    ms, tot, _ = timed_run(args.alpha)
+    clocks = sampler.stop() if sampler else None
+    ms = max_over_ranks(ms)
+    value = world * BATCH * K / (ms / 1e3)
+
+    # ---- the same kernels at alpha = 1 (full depth) and 0.999
+    others = {}
+    for a in (1.0, 0.999):
+        if abs(a - args.alpha) < 1e-12:
+            continue
+        ms_a, tot_a, _ = timed_run(a)
+        ms_a = max_over_ranks(ms_a)
+        others[a] = (ms_a, tot_a)
+
+    # ---- per-kernel-class device times of the same K steps (events around each launch)
+    _, _, prof = timed_run(args.alpha, profile=True)
+
+    # ---- end to end through the C ABI: host token in, argmax token out, every step
+    model.d3_reset_slot(0)
+    model.d3_prefill(0, prompt)
+    tok_dev = torch.empty(BATCH, dtype=torch.int32, device=dev)
+    tok_host = torch.empty(BATCH, dtype=torch.int32).pin_memory()
+    cur = int(toks[0])
+    for j in range(W):
+        model.d3_decode_step([0], [cur], [gi[0]], args.alpha, logits=logits)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record(stream)
+    for j in range(K):
+        model.d3_decode_step([0], [cur], [gi[j]], args.alpha, logits=logits)   # host arrays -> device
+        model.d3_argmax(logits, tok_dev)
+        tok_host.copy_(tok_dev, non_blocking=True)                              # device -> host
+        stream.synchronize()
+        cur = int(tok_host[0])
+    e1.record(stream)
+    barrier()
+    e2e_ms = max_over_ranks(e0.elapsed_time(e1))
+    e2e_value = world * BATCH * K / (e2e_ms / 1e3)
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return 0
+
+    peak, peak_kind = measured_peak()
+    # dominant kernel class and its algorithmic bytes per launch
+    d, f = shape.d_model, shape.d_ffn
+    nq = shape.n_q_heads * shape.head_dim
+    class_bytes = {
+        "norm+qkv": 2 * shape.qkv_rows * d + 2 * d + 4 * d + 4 * shape.qkv_rows,
+        "o_proj+resid": 2 * d * nq + 4 * nq + 8 * d,
+        "norm+gate_up+swiglu": 2 * 2 * f * d + 2 * d + 4 * d + 4 * f,
+        "down+resid": 2 * d * f + 4 * f + 8 * d,
+        "norm+lm_head": 2 * shape.vocab * d + 2 * d + 4 * d + 4 * shape.vocab,
+    }
+    top = max(prof.items(), key=lambda kv: kv[1]["ms"])
+    top_name, top_ms, top_n = top[0], top[1]["ms"], top[1]["launches"]
+    prof_total = sum(v["ms"] for v in prof.values())
+    roofline = {"bound": "hbm", "kernel": top_name, "unit": "GB/s", "peak": peak,
+                "peak_kind": f"of {peak_kind} (STREAM-style copy)", "traffic": None,
+                "share_of_kernel_time": top_ms / prof_total, "launches": top_n}
+    if top_name in class_bytes:
+        ach = class_bytes[top_name] * BATCH / 1e9 / (top_ms / top_n / 1e3)
+        roofline.update(achieved=ach, frac=ach / peak, bytes_per_launch=class_bytes[top_name],
+                        avg_launch_us=1e3 * top_ms / top_n)
+    else:
+        roofline.update(achieved=None, frac=None)
+    step_gbs = tot["bytes"] / 1e9 / (ms / 1e3)
+    step_roofline = {"bytes_per_step": tot["bytes"] / K, "achieved": step_gbs, "unit": "GB/s",
+                     "frac_of_measured": step_gbs / peak, "frac_of_nominal_8TBs": step_gbs / NOMINAL_HBM_GBS,
+                     "avg_layers_per_token": tot["rows_layers"] / K}
+    alphas = {str(args.alpha): {"tokens_per_s": value, "ms_per_step": ms / K,
+                                "avg_layers": tot["rows_layers"] / K,
+                                "frac_of_measured": step_gbs / peak}}
+    for a, (ms_a, tot_a) in others.items():
+        g = tot_a["bytes"] / 1e9 / (ms_a / 1e3)
+        alphas[str(a)] = {"tokens_per_s": world * BATCH * K / (ms_a / 1e3), "ms_per_step": ms_a / K,
+                          "avg_layers": tot_a["rows_layers"] / K, "frac_of_measured": g / peak}
+    if 1.0 in others:
+        full = alphas["1.0"]
+        alphas["speedup_vs_alpha_1"] = value / full["tokens_per_s"]
+        alphas["layer_ratio_vs_alpha_1"] = full["avg_layers"] / (tot["rows_layers"] / K)
+        alphas["bytes_ratio_vs_alpha_1"] = others[1.0][1]["bytes"] / tot["bytes"]
+
+    cpu_baseline = None
+    if world == 1 and not args.no_cpu_baseline:
+        oshape, scale, note = oracle_shape_and_scale(shape)
+        w_cpu = I.weights_to({k: (v[:oshape.n_layers] if isinstance(v, list) else v)
+                              for k, v in w.items()}, "cpu")
+        tps, dt, cores = time_oracle(oshape, w_cpu, args.alpha, start_id, 16, 1)
+        cpu_baseline = {"value": tps * scale, "unit": "tokens/s", "cores": cores, "kind": "oracle",
+                        "sample": f"fp64 C oracle, 7B shape, {note}, prompt {ORACLE_PROMPT}, 16 decode "
+                                  f"steps at alpha={args.alpha}, {dt:.1f} s of CPU work"}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": K,
+        "warmup": W, "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16 weights+KV, f32 activations/accumulate", "data": "synthetic",
+        "config": {"workload": f"llama2-7b-shape (L={shape.n_layers},d=4096,32x128,ffn 11008,V=32000), "
+                               f"batch 1, prompt {args.prompt}, generate 256", "alpha": args.alpha, "start_id": start_id,
+                   "anchor": "start", "kv_fill": "copy", "gen_index_schedule": "1 + floor(j*255/K)",
+                   "l2": "inputs_exceed_l2 (weights of one step >> 126 MB)",
+                   "multi_gpu": "independent replicas"},
+        "roofline": roofline, "step_roofline": step_roofline, "alphas": alphas,
+        "kernel_classes": prof, "cpu_baseline": cpu_baseline,
+        "e2e": {"value": e2e_value, "unit": "tokens/s", "ms_per_step": e2e_ms / K,
+                "h2d_bytes_per_step": 12 * BATCH, "d2h_bytes_per_step": 4 * BATCH},
+        "gpu_launches": tot["launches"], "clocks": clocks,
+    }
+    print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.destroy_process_group()
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())

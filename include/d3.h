@@ -164,6 +164,17 @@ int32_t d3_read_hidden(d3_model *m, float *hidden);
 /* one KV-cache entry to HOST: k, v [Hkv * head_dim] fp32 */
 int32_t d3_read_kv(d3_model *m, int32_t layer, int32_t slot, int32_t pos, float *k, float *v);
 
+/* Per-kernel-class device times (measurement aid for Sec. 4.2-style wall-clock
+ * accounting).  While enabled, every step records CUDA events around each of its
+ * launches on the model's stream and waits for the step to finish, so enabled
+ * steps are slower end to end; totals accumulate until read.
+ * d3_read_profile: ms[k], launches[k] for k < D3_PROF_KINDS (HOST arrays), then
+ * clears the totals.  d3_profile_name(k): a static string. */
+#define D3_PROF_KINDS 10
+int32_t d3_profile(d3_model *m, int32_t enable);
+int32_t d3_read_profile(d3_model *m, float *ms, int32_t *launches);
+const char *d3_profile_name(int32_t kind);
+
 int32_t d3_slot_pos(const d3_model *m, int32_t slot); /* tokens cached; D3_ESTATE if never prefilled */
 int32_t d3_reset_slot(d3_model *m, int32_t slot);
 int32_t d3_sync(d3_model *m); /* wait for the stream; returns a deferred device status */

@@ -18,11 +18,11 @@ from . import build as _build
 OK, EINVAL, ECAPACITY, ESTATE, ECUDA, ETIMEOUT = 0, -1, -2, -3, -4, -5
 ANCHOR_START, ANCHOR_TAIL = 0, 1
 FILL_NONE, FILL_COPY, FILL_RECOMPUTE = 0, 1, 2
-MAX_BATCH, MAX_LAYERS = 64, 128
+MAX_BATCH, MAX_LAYERS, PROF_KINDS = 64, 128, 10
 
 EXPORTS = ("d3_depth", "d3_schedule", "d3_workspace_bytes", "d3_load", "d3_prefill",
            "d3_decode_step", "d3_argmax", "d3_read_schedule", "d3_read_hidden", "d3_read_kv",
-           "d3_slot_pos", "d3_reset_slot", "d3_sync", "d3_free", "d3_strerror")
+           "d3_profile", "d3_read_profile", "d3_profile_name", "d3_slot_pos", "d3_reset_slot", "d3_sync", "d3_free", "d3_strerror")
 
 
 class Config(C.Structure):
@@ -69,6 +69,10 @@ def _load() -> C.CDLL:
     lib.d3_read_schedule.argtypes = [P, P, P, P, P]
     lib.d3_read_hidden.argtypes = [P, P]
     lib.d3_read_kv.argtypes = [P, I32, I32, I32, P, P]
+    lib.d3_profile.argtypes = [P, I32]
+    lib.d3_read_profile.argtypes = [P, P, P]
+    lib.d3_profile_name.argtypes = [I32]
+    lib.d3_profile_name.restype = C.c_char_p
     lib.d3_slot_pos.argtypes = [P, I32]
     lib.d3_reset_slot.argtypes = [P, I32]
     lib.d3_sync.argtypes = [P]
@@ -246,6 +250,21 @@ class D3Model:
         if rc != OK:
             raise D3Error(rc, "d3_read_kv")
         return k, v
+
+    def d3_profile(self, enable: bool) -> None:
+        rc = LIB.d3_profile(self.h, int(enable))
+        if rc != OK:
+            raise D3Error(rc, "d3_profile")
+
+    def d3_read_profile(self) -> Dict[str, Dict[str, float]]:
+        """{kernel class: {"ms": total device ms, "launches": count}} since the last read."""
+        ms = np.zeros(PROF_KINDS, np.float32)
+        cnt = np.zeros(PROF_KINDS, np.int32)
+        rc = LIB.d3_read_profile(self.h, ms.ctypes.data, cnt.ctypes.data)
+        if rc != OK:
+            raise D3Error(rc, "d3_read_profile")
+        return {LIB.d3_profile_name(k).decode(): {"ms": float(ms[k]), "launches": int(cnt[k])}
+                for k in range(PROF_KINDS) if cnt[k] > 0}
 
     def d3_slot_pos(self, slot: int) -> int:
         return int(LIB.d3_slot_pos(self.h, slot))

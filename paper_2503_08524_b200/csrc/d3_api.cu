@@ -88,6 +88,12 @@ struct d3_model {
   int32_t last_B;
   int32_t last_perm[D3_MAX_BATCH];
   int64_t layer_bytes, head_bytes;
+  // per-kernel-class timing (d3_profile)
+  bool prof_on;
+  std::vector<cudaEvent_t> prof_events;   // pool, two per recorded launch
+  std::vector<int> prof_kind;             // kind of each recorded pair of the running step
+  float prof_ms[D3_PROF_KINDS];
+  int32_t prof_n[D3_PROF_KINDS];
 
   DevSched *sched() const { return reinterpret_cast<DevSched *>(scratch + lay.sched); }
   float2 *rope() const { return reinterpret_cast<float2 *>(scratch + lay.rope); }
@@ -98,6 +104,46 @@ struct d3_model {
   float *part_ml() const { return reinterpret_cast<float *>(scratch + lay.part_ml); }
   float *u() const { return reinterpret_cast<float *>(scratch + lay.u); }
 };
+
+enum ProfKind { PK_SCHED = 0, PK_QKV, PK_ROPE, PK_ATTN, PK_OPROJ, PK_GATEUP, PK_DOWN, PK_FILL,
+                PK_HEAD, PK_OTHER };
+static const char *kProfNames[D3_PROF_KINDS] = {"schedule+embed", "norm+qkv", "rope+kv_append",
+                                                "attention", "o_proj+resid", "norm+gate_up+swiglu",
+                                                "down+resid", "kv_fill", "norm+lm_head", "other"};
+
+// Scope that brackets one launch (or a launcher's pair of launches) with events.
+struct ProfScope {
+  d3_model *m;
+  cudaEvent_t stop;
+  ProfScope(d3_model *mm, int kind) : m(mm), stop(nullptr) {
+    if (!m->prof_on) return;
+    size_t i = m->prof_kind.size() * 2;
+    while (m->prof_events.size() < i + 2) {
+      cudaEvent_t e;
+      if (cudaEventCreate(&e) != cudaSuccess) return;
+      m->prof_events.push_back(e);
+    }
+    m->prof_kind.push_back(kind);
+    cudaEventRecord(m->prof_events[i], m->stream);
+    stop = m->prof_events[i + 1];
+  }
+  ~ProfScope() {
+    if (stop) cudaEventRecord(stop, m->stream);
+  }
+};
+
+static void prof_collect(d3_model *m) {
+  if (!m->prof_on) return;
+  cudaStreamSynchronize(m->stream);
+  for (size_t i = 0; i < m->prof_kind.size(); ++i) {
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, m->prof_events[2 * i], m->prof_events[2 * i + 1]) == cudaSuccess) {
+      m->prof_ms[m->prof_kind[i]] += ms;
+      m->prof_n[m->prof_kind[i]] += 1;
+    }
+  }
+  m->prof_kind.clear();
+}
 
 static const int32_t *thr_for(d3_model *m, double alpha) {
   uint64_t key;
@@ -123,7 +169,7 @@ static int32_t run_step(d3_model *m, const StepArgs &a, const int32_t *n, const 
   cudaStream_t st = m->stream;
   const int B = a.B, L = c.n_layers;
   int launches = 0;
-  launches += launch_schedule_embed(a, m->sched(), m->embed, m->x(), dm.d, st);
+  { ProfScope ps(m, PK_SCHED); launches += launch_schedule_embed(a, m->sched(), m->embed, m->x(), dm.d, st); }
   const int nq = dm.Hq * dm.dh, nkv = dm.Hkv * dm.dh;
   const int G = dm.Hq / dm.Hkv, GQ = (G % 4 == 0) ? 4 : (G % 2 == 0) ? 2 : 1;
 
@@ -140,9 +186,10 @@ static int32_t run_step(d3_model *m, const StepArgs &a, const int32_t *n, const 
       g.W = m->wqkv[l]; g.W2 = nullptr; g.R = dm.qkv_rows; g.K = dm.d;
       g.act = m->x(); g.act_stride = dm.d; g.gain = m->attn_norm[l];
       g.out = m->qkv(); g.out_stride = dm.qkv_rows; g.out_col0 = 0;
-      launches += launch_gemv(g, EPI_STORE, ml, st);
-      launches += launch_rope_append(m->qkv(), m->rope(), m->Kc, m->Vc, m->sched(), l, ROWS_PREFIX,
-                                     0, ml, dm, st);
+      { ProfScope ps(m, PK_QKV); launches += launch_gemv(g, EPI_STORE, ml, st); }
+      { ProfScope ps(m, PK_ROPE);
+        launches += launch_rope_append(m->qkv(), m->rope(), m->Kc, m->Vc, m->sched(), l, ROWS_PREFIX,
+                                       0, ml, dm, st); }
       // attention over the cache (positions 0..pos, the new one included)
       int max_len = 1;
       for (int r = 0; r < ml; ++r) {
@@ -156,20 +203,21 @@ static int32_t run_step(d3_model *m, const StepArgs &a, const int32_t *n, const 
       int split_len = ((max_len + want - 1) / want + 31) / 32 * 32;
       if (split_len < 32) split_len = 32;
       int n_splits = (max_len + split_len - 1) / split_len;
-      launches += launch_attention(m->qkv(), m->Kc, m->Vc, m->sched(), l, ml, split_len, n_splits,
-                                   m->lay.max_splits, m->part_o(), m->part_ml(), m->attn_out(), dm, st);
+      { ProfScope ps(m, PK_ATTN);
+        launches += launch_attention(m->qkv(), m->Kc, m->Vc, m->sched(), l, ml, split_len, n_splits,
+                                     m->lay.max_splits, m->part_o(), m->part_ml(), m->attn_out(), dm, st); }
       // output projection + residual
       g.W = m->wo[l]; g.R = dm.d; g.K = nq; g.act = m->attn_out(); g.act_stride = nq;
       g.gain = nullptr; g.out = m->x(); g.out_stride = dm.d;
-      launches += launch_gemv(g, EPI_RESID, ml, st);
+      { ProfScope ps(m, PK_OPROJ); launches += launch_gemv(g, EPI_RESID, ml, st); }
       // RMSNorm + gate/up + SiLU * mul
       g.W = m->w_gate[l]; g.W2 = m->w_up[l]; g.R = dm.f; g.K = dm.d; g.act = m->x();
       g.act_stride = dm.d; g.gain = m->mlp_norm[l]; g.out = m->u(); g.out_stride = dm.f;
-      launches += launch_gemv(g, EPI_SWIGLU, ml, st);
+      { ProfScope ps(m, PK_GATEUP); launches += launch_gemv(g, EPI_SWIGLU, ml, st); }
       // down projection + residual
       g.W = m->w_down[l]; g.W2 = nullptr; g.R = dm.d; g.K = dm.f; g.act = m->u();
       g.act_stride = dm.f; g.gain = nullptr; g.out = m->x(); g.out_stride = dm.d;
-      launches += launch_gemv(g, EPI_RESID, ml, st);
+      { ProfScope ps(m, PK_DOWN); launches += launch_gemv(g, EPI_RESID, ml, st); }
     }
     if (c.kv_fill == D3_FILL_RECOMPUTE && ml < B) {
       // rows that drop block l: K,V from the block's own norm, W_k, W_v on the carried state
@@ -177,6 +225,7 @@ static int32_t run_step(d3_model *m, const StepArgs &a, const int32_t *n, const 
       g.W = m->wqkv[l] + (size_t)nq * dm.d; g.W2 = nullptr; g.R = 2 * nkv; g.K = dm.d;
       g.act = m->x(); g.act_stride = dm.d; g.gain = m->attn_norm[l];
       g.out = m->qkv(); g.out_stride = dm.qkv_rows; g.out_col0 = nq;
+      ProfScope ps(m, PK_FILL);
       launches += launch_gemv(g, EPI_STORE, B - ml, st);
       launches += launch_rope_append(m->qkv(), m->rope(), m->Kc, m->Vc, m->sched(), l, ROWS_SUFFIX,
                                      1, B - ml, dm, st);
@@ -186,17 +235,18 @@ static int32_t run_step(d3_model *m, const StepArgs &a, const int32_t *n, const 
   if (c.kv_fill == D3_FILL_COPY) {
     bool any = false;
     for (int b = 0; b < B; ++b) any = any || hi[b] > lo[b];
-    if (any) launches += launch_fill_copy(m->Kc, m->Vc, m->sched(), B, dm, st);
+    if (any) { ProfScope ps(m, PK_FILL); launches += launch_fill_copy(m->Kc, m->Vc, m->sched(), B, dm, st); }
   }
   if (logits_dev) {
     g.layer = 0; g.row_mode = logits_mode;
     g.W = m->lm_head; g.W2 = nullptr; g.R = dm.V; g.K = dm.d; g.act = m->x(); g.act_stride = dm.d;
     g.gain = m->final_norm; g.out = logits_dev; g.out_stride = dm.V; g.out_col0 = 0;
-    launches += launch_gemv(g, EPI_LOGITS, logits_mode == ROWS_LAST ? 1 : B, st);
+    { ProfScope ps(m, PK_HEAD); launches += launch_gemv(g, EPI_LOGITS, logits_mode == ROWS_LAST ? 1 : B, st); }
   }
   m->last_B = B;
   for (int b = 0; b < B; ++b) m->last_perm[b] = perm[b];
   (void)n;
+  prof_collect(m);
   if (launches_out) *launches_out = launches;
   return cudaGetLastError() == cudaSuccess ? D3_OK : D3_ECUDA;
 }
@@ -298,6 +348,9 @@ int32_t d3_load(const d3_config *cfg, const d3_weights *w, void *kv_dev, void *s
   m->scratch = (char *)scratch_dev;
   m->pos.assign(cfg->max_slots, -1);
   m->last_B = 0;
+  m->prof_on = false;
+  memset(m->prof_ms, 0, sizeof(m->prof_ms));
+  memset(m->prof_n, 0, sizeof(m->prof_n));
   const int64_t d = cfg->d_model, f = cfg->d_ffn;
   m->layer_bytes = 2 * ((int64_t)m->dm.qkv_rows * d + d * cfg->n_q_heads * cfg->head_dim + 3 * d * f + 2 * d);
   m->head_bytes = 2 * ((int64_t)cfg->vocab * d + d);
@@ -465,7 +518,30 @@ int32_t d3_sync(d3_model *m) {
   return status;
 }
 
-void d3_free(d3_model *m) { delete m; }
+int32_t d3_profile(d3_model *m, int32_t enable) {
+  if (!m) return D3_EINVAL;
+  m->prof_on = enable != 0;
+  return D3_OK;
+}
+
+int32_t d3_read_profile(d3_model *m, float *ms, int32_t *launches) {
+  if (!m || !ms || !launches) return D3_EINVAL;
+  memcpy(ms, m->prof_ms, sizeof(m->prof_ms));
+  memcpy(launches, m->prof_n, sizeof(m->prof_n));
+  memset(m->prof_ms, 0, sizeof(m->prof_ms));
+  memset(m->prof_n, 0, sizeof(m->prof_n));
+  return D3_OK;
+}
+
+const char *d3_profile_name(int32_t kind) {
+  return (kind >= 0 && kind < D3_PROF_KINDS) ? kProfNames[kind] : "";
+}
+
+void d3_free(d3_model *m) {
+  if (!m) return;
+  for (cudaEvent_t e : m->prof_events) cudaEventDestroy(e);
+  delete m;
+}
 
 const char *d3_strerror(int32_t code) {
   switch (code) {
