@@ -164,6 +164,14 @@ int32_t d3_read_hidden(d3_model *m, float *hidden);
 /* one KV-cache entry to HOST: k, v [Hkv * head_dim] fp32 */
 int32_t d3_read_kv(d3_model *m, int32_t layer, int32_t slot, int32_t pos, float *k, float *v);
 
+/* How decode steps execute.  AUTO: a batch of one row runs as a single persistent
+ * cooperative kernel when the device and sizes allow it (fill modes NONE and
+ * COPY), everything else as a sequence of kernels per block.  KERNELS: always the
+ * sequence of kernels.  Both compute the same step (Sec. 3.4). */
+#define D3_EXEC_AUTO 0
+#define D3_EXEC_KERNELS 1
+int32_t d3_set_exec(d3_model *m, int32_t mode);
+
 /* Per-kernel-class device times (measurement aid for Sec. 4.2-style wall-clock
  * accounting).  While enabled, every step records CUDA events around each of its
  * launches on the model's stream and waits for the step to finish, so enabled

@@ -19,10 +19,11 @@ OK, EINVAL, ECAPACITY, ESTATE, ECUDA, ETIMEOUT = 0, -1, -2, -3, -4, -5
 ANCHOR_START, ANCHOR_TAIL = 0, 1
 FILL_NONE, FILL_COPY, FILL_RECOMPUTE = 0, 1, 2
 MAX_BATCH, MAX_LAYERS, PROF_KINDS = 64, 128, 10
+EXEC_AUTO, EXEC_KERNELS = 0, 1
 
 EXPORTS = ("d3_depth", "d3_schedule", "d3_workspace_bytes", "d3_load", "d3_prefill",
            "d3_decode_step", "d3_argmax", "d3_read_schedule", "d3_read_hidden", "d3_read_kv",
-           "d3_profile", "d3_read_profile", "d3_profile_name", "d3_slot_pos", "d3_reset_slot", "d3_sync", "d3_free", "d3_strerror")
+           "d3_set_exec", "d3_profile", "d3_read_profile", "d3_profile_name", "d3_slot_pos", "d3_reset_slot", "d3_sync", "d3_free", "d3_strerror")
 
 
 class Config(C.Structure):
@@ -69,6 +70,7 @@ def _load() -> C.CDLL:
     lib.d3_read_schedule.argtypes = [P, P, P, P, P]
     lib.d3_read_hidden.argtypes = [P, P]
     lib.d3_read_kv.argtypes = [P, I32, I32, I32, P, P]
+    lib.d3_set_exec.argtypes = [P, I32]
     lib.d3_profile.argtypes = [P, I32]
     lib.d3_read_profile.argtypes = [P, P, P]
     lib.d3_profile_name.argtypes = [I32]
@@ -250,6 +252,11 @@ class D3Model:
         if rc != OK:
             raise D3Error(rc, "d3_read_kv")
         return k, v
+
+    def d3_set_exec(self, mode: int) -> None:
+        rc = LIB.d3_set_exec(self.h, mode)
+        if rc != OK:
+            raise D3Error(rc, "d3_set_exec")
 
     def d3_profile(self, enable: bool) -> None:
         rc = LIB.d3_profile(self.h, int(enable))

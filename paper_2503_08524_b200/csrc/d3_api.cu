@@ -27,6 +27,10 @@ Layout make_layout(const d3_config &c) {
   y.part_o = off;   off = align_up(off + B * c.n_q_heads * y.max_splits * c.head_dim * 4, 256);
   y.part_ml = off;  off = align_up(off + B * c.n_q_heads * y.max_splits * 2 * 4, 256);
   y.u = off;        off = align_up(off + B * c.d_ffn * 4, 256);
+  y.layer_tab = off; off = align_up(off + (size_t)c.n_layers * sizeof(LayerPtrs), 256);
+  y.bar = off;      off = align_up(off + 256, 256);
+  y.part_fused = off;
+  off = align_up(off + (size_t)c.n_q_heads * kFusedMaxCtas * (c.head_dim + 2) * 4, 256);
   y.total = off;
   return y;
 }
@@ -94,6 +98,12 @@ struct d3_model {
   std::vector<int> prof_kind;             // kind of each recorded pair of the running step
   float prof_ms[D3_PROF_KINDS];
   int32_t prof_n[D3_PROF_KINDS];
+  // fused batch-1 step kernel
+  int32_t exec_mode;
+  int fused_ok, fused_grid, fused_stages, fused_act;
+  size_t fused_smem;
+  void *fused_func;
+  std::vector<LayerPtrs> layer_tab_host;
 
   DevSched *sched() const { return reinterpret_cast<DevSched *>(scratch + lay.sched); }
   float2 *rope() const { return reinterpret_cast<float2 *>(scratch + lay.rope); }
@@ -106,10 +116,10 @@ struct d3_model {
 };
 
 enum ProfKind { PK_SCHED = 0, PK_QKV, PK_ROPE, PK_ATTN, PK_OPROJ, PK_GATEUP, PK_DOWN, PK_FILL,
-                PK_HEAD, PK_OTHER };
+                PK_HEAD, PK_FUSED };
 static const char *kProfNames[D3_PROF_KINDS] = {"schedule+embed", "norm+qkv", "rope+kv_append",
                                                 "attention", "o_proj+resid", "norm+gate_up+swiglu",
-                                                "down+resid", "kv_fill", "norm+lm_head", "other"};
+                                                "down+resid", "kv_fill", "norm+lm_head", "fused_step"};
 
 // Scope that brackets one launch (or a launcher's pair of launches) with events.
 struct ProfScope {
@@ -251,6 +261,35 @@ static int32_t run_step(d3_model *m, const StepArgs &a, const int32_t *n, const 
   return cudaGetLastError() == cudaSuccess ? D3_OK : D3_ECUDA;
 }
 
+// One batch-1 step as a single cooperative kernel.
+static int32_t run_fused_step(d3_model *m, const StepArgs &a, float *logits_dev, int32_t *launches_out) {
+  FusedParams fp;
+  memset(&fp, 0, sizeof(fp));
+  fp.slot = a.slot[0]; fp.tok = a.tok[0]; fp.gi = a.gi[0]; fp.pos = a.pos[0]; fp.tok_dev = a.tok_dev;
+  memcpy(fp.thr, a.thr, sizeof(fp.thr));
+  fp.L = a.L; fp.start_id = a.start_id; fp.anchor = a.anchor; fp.kv_fill = m->cfg.kv_fill;
+  fp.dm = m->dm; fp.eps = m->cfg.rms_eps;
+  fp.layers = reinterpret_cast<const LayerPtrs *>(m->scratch + m->lay.layer_tab);
+  fp.embed = m->embed; fp.lm_head = m->lm_head; fp.final_norm = m->final_norm;
+  fp.Kc = m->Kc; fp.Vc = m->Vc; fp.rope = m->rope(); fp.sched = m->sched();
+  fp.bar_counter = reinterpret_cast<unsigned *>(m->scratch + m->lay.bar);
+  fp.x = m->x(); fp.qkv = m->qkv(); fp.u = m->u();
+  fp.part = reinterpret_cast<float *>(m->scratch + m->lay.part_fused);
+  fp.logits = logits_dev;
+  fp.n_stages = m->fused_stages; fp.act_floats = m->fused_act;
+  fp.wait_ns = 2000000000ull;
+  int rc;
+  {
+    ProfScope ps(m, PK_FUSED);
+    rc = launch_fused_step(m->fused_func, m->fused_grid, m->fused_smem, fp, m->stream);
+  }
+  m->last_B = 1;
+  m->last_perm[0] = 0;
+  prof_collect(m);
+  if (launches_out) *launches_out = 1;
+  return (rc == 1 && cudaGetLastError() == cudaSuccess) ? D3_OK : D3_ECUDA;
+}
+
 extern "C" {
 
 int32_t d3_depth(int32_t L, double alpha, int64_t i) {
@@ -355,6 +394,18 @@ int32_t d3_load(const d3_config *cfg, const d3_weights *w, void *kv_dev, void *s
   m->layer_bytes = 2 * ((int64_t)m->dm.qkv_rows * d + d * cfg->n_q_heads * cfg->head_dim + 3 * d * f + 2 * d);
   m->head_bytes = 2 * ((int64_t)cfg->vocab * d + d);
   if (init_kernel_attributes() != 0) { delete m; return D3_ECUDA; }
+  m->exec_mode = D3_EXEC_AUTO;
+  for (int l = 0; l < L; ++l)
+    m->layer_tab_host.push_back(LayerPtrs{m->attn_norm[l], m->wqkv[l], m->wo[l], m->mlp_norm[l],
+                                          m->w_gate[l], m->w_up[l], m->w_down[l]});
+  if (cudaMemcpyAsync(m->scratch + m->lay.layer_tab, m->layer_tab_host.data(),
+                      sizeof(LayerPtrs) * L, cudaMemcpyHostToDevice, m->stream) != cudaSuccess) {
+    delete m;
+    return D3_ECUDA;
+  }
+  m->fused_ok = fused_plan(*cfg, &m->fused_grid, &m->fused_stages, &m->fused_act, &m->fused_smem,
+                           &m->fused_func);
+  if (m->fused_ok && m->fused_grid > kFusedMaxCtas) m->fused_grid = kFusedMaxCtas;
   if (cudaMemsetAsync(m->sched(), 0, sizeof(DevSched), m->stream) != cudaSuccess) { delete m; return D3_ECUDA; }
   launch_rope_table(m->rope(), cfg->max_seq, cfg->head_dim, cfg->rope_base, m->stream);
   if (cudaGetLastError() != cudaSuccess) { delete m; return D3_ECUDA; }
@@ -424,7 +475,10 @@ int32_t d3_decode_step(d3_model *m, int32_t batch, const int32_t *slots, const i
                            &rows_layers, &touched);
   if (rc != D3_OK) return rc;
   int32_t launches = 0;
-  rc = run_step(m, a, n, lo, hi, perm, m_l, logits_dev, ROWS_ALL, &launches);
+  const bool fused = batch == 1 && m->fused_ok && m->exec_mode == D3_EXEC_AUTO &&
+                     c.kv_fill != D3_FILL_RECOMPUTE;
+  rc = fused ? run_fused_step(m, a, logits_dev, &launches)
+             : run_step(m, a, n, lo, hi, perm, m_l, logits_dev, ROWS_ALL, &launches);
   if (rc != D3_OK) return rc;
   if (stats) {
     if (stats->n) memcpy(stats->n, n, sizeof(int32_t) * batch);
@@ -516,6 +570,12 @@ int32_t d3_sync(d3_model *m) {
   if (cudaMemcpy(&status, &m->sched()->status, 4, cudaMemcpyDeviceToHost) != cudaSuccess)
     return D3_ECUDA;
   return status;
+}
+
+int32_t d3_set_exec(d3_model *m, int32_t mode) {
+  if (!m || (mode != D3_EXEC_AUTO && mode != D3_EXEC_KERNELS)) return D3_EINVAL;
+  m->exec_mode = mode;
+  return D3_OK;
 }
 
 int32_t d3_profile(d3_model *m, int32_t enable) {

@@ -1,0 +1,795 @@
+// Batch-1 decode step as ONE persistent cooperative kernel (sm_100a).
+//
+// One CTA per SM.  Warp 8 is the producer: a single thread streams the CTA's
+// share of every weight matrix (and of the static part of the KV cache) through
+// a shared-memory ring with bulk asynchronous copies (cp.async.bulk + mbarrier
+// transaction counts).  It never waits for the computation, so HBM stays busy
+// across phase boundaries: weights do not depend on activations.  Warps 0-7
+// consume ring stages in lockstep.  Phases of a block (RMSNorm+QKV+RoPE+KV
+// append | attention | O-proj+residual | RMSNorm+gate/up+SwiGLU | down+residual)
+// are separated by grid barriers on a global counter; only the small fp32
+// activations cross them (through L2, read with ld.global.cg).
+//
+// A ring stage is 16 KB: four weight-row segments of 2048 bf16 (a "row group" x
+// k-chunk), or 8 KB of K plus 8 KB of V for one KV head.  In a GEMV stage thread
+// t owns k = t*8..t*8+7 of the chunk for all four rows, so the activation costs
+// two shared loads per four weight loads.
+//
+// Every wait (mbarrier, grid barrier) is bounded; on expiry the kernel raises
+// D3_ETIMEOUT in the schedule's status word, stops issuing copies, drains the
+// copies in flight and returns.
+#include "d3_internal.cuh"
+
+namespace d3 {
+
+namespace {
+
+constexpr int kConsumers = 256;
+constexpr int kFusedThreads = 288;
+constexpr int kStageBytes = 16384;
+constexpr int kChunk = 2048;          // weight elements of one row segment
+constexpr int kMaxStages = 14;
+constexpr int kMaxGQ = 4;
+
+enum PhaseKind { PH_QKV = 0, PH_OPROJ, PH_GATEUP, PH_DOWN, PH_HEAD };
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) {
+  return (uint32_t)__cvta_generic_to_shared(p);
+}
+__device__ __forceinline__ float bfl(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bfh(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok;
+}
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+      "l"(src), "r"(bytes), "r"(bar)
+      : "memory");
+}
+__device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+
+__device__ __forceinline__ float4 ldcg4(const float *p) { return __ldcg(reinterpret_cast<const float4 *>(p)); }
+
+}  // namespace
+
+
+namespace {
+
+struct Ctx {
+  const FusedParams *p;
+  unsigned char *ring;
+  float *act;
+  uint64_t *full, *empty;
+  volatile int *abort_flag;
+  float (*red)[8][4];
+  int cta, ncta;
+};
+
+// ---- bounded waits ---------------------------------------------------------
+__device__ __forceinline__ uint64_t now_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+
+// Wait for an mbarrier phase for at most wait_ns.  Returns false at once when
+// the CTA is in abort mode, or after raising D3_ETIMEOUT and entering it.
+__device__ __forceinline__ bool wait_bar(const Ctx &c, uint32_t bar, uint32_t parity) {
+  if (*c.abort_flag) return false;
+  if (mbar_try_wait(bar, parity)) return true;
+  const uint64_t t0 = now_ns();
+  for (uint32_t it = 1;; ++it) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((it & 63u) == 0u) {
+      if (*c.abort_flag) return false;
+      if (now_ns() - t0 > c.p->wait_ns) break;
+    }
+  }
+  c.p->sched->status = D3_ETIMEOUT;
+  *c.abort_flag = 1;
+  return false;
+}
+
+// Grid barrier number `idx` (1-based) among the consumer threads of all CTAs.
+__device__ __forceinline__ bool grid_barrier(const Ctx &c, unsigned idx) {
+  consumer_sync();
+  if (threadIdx.x == 0) {
+    __threadfence();
+    atomicAdd(c.p->bar_counter, 1u);
+    const unsigned target = idx * (unsigned)c.ncta;
+    const uint64_t t0 = now_ns();
+    for (uint32_t it = 1; !*c.abort_flag; ++it) {
+      unsigned v;
+      asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(c.p->bar_counter) : "memory");
+      if (v >= target) break;
+      if ((it & 15u) == 0u && now_ns() - t0 > c.p->wait_ns) {
+        c.p->sched->status = D3_ETIMEOUT;
+        *c.abort_flag = 1;
+      }
+    }
+    __threadfence();
+  }
+  consumer_sync();
+  return *c.abort_flag == 0;
+}
+
+// ---- the CTA's share of a phase ---------------------------------------------
+struct Phase {
+  int kind;
+  const bf16 *W, *W2;
+  int K, R;          // row length, rows of W
+  int groups;        // row groups of the phase
+  int g0, g1;        // this CTA's groups
+  int nkc;           // k-chunks per row
+};
+
+__device__ __forceinline__ void split_range(int total, int cta, int ncta, int &b, int &e) {
+  b = (int)(((long long)total * cta) / ncta);
+  e = (int)(((long long)total * (cta + 1)) / ncta);
+}
+
+__device__ __forceinline__ Phase make_phase(const FusedParams &p, int kind, int layer, int cta, int ncta) {
+  Phase ph;
+  ph.kind = kind;
+  ph.W2 = nullptr;
+  const Dims &dm = p.dm;
+  if (kind == PH_QKV) { ph.W = p.layers[layer].wqkv; ph.K = dm.d; ph.R = dm.qkv_rows; ph.groups = dm.qkv_rows / 4; }
+  else if (kind == PH_OPROJ) { ph.W = p.layers[layer].wo; ph.K = dm.Hq * dm.dh; ph.R = dm.d; ph.groups = dm.d / 4; }
+  else if (kind == PH_GATEUP) { ph.W = p.layers[layer].w_gate; ph.W2 = p.layers[layer].w_up; ph.K = dm.d; ph.R = dm.f; ph.groups = dm.f / 2; }
+  else if (kind == PH_DOWN) { ph.W = p.layers[layer].w_down; ph.K = dm.f; ph.R = dm.d; ph.groups = dm.d / 4; }
+  else { ph.W = p.lm_head; ph.K = dm.d; ph.R = dm.V; ph.groups = (dm.V + 3) / 4; }
+  split_range(ph.groups, cta, ncta, ph.g0, ph.g1);
+  ph.nkc = (ph.K + kChunk - 1) / kChunk;
+  return ph;
+}
+
+// the four weight rows of group g (row pointers; rows beyond R are clamped)
+__device__ __forceinline__ void group_rows(const Phase &ph, const Dims &dm, int g, const bf16 *rows[4], int ridx[4]) {
+  if (ph.kind == PH_QKV) {
+    const int per_head = dm.dh / 4, half = dm.dh / 2;
+    const int rot_groups = (dm.Hq + dm.Hkv) * per_head;
+    if (g < rot_groups) {   // q or k head: two rotary pairs (j, j+half), (j+1, j+1+half)
+      int head = g / per_head, jj = (g % per_head) * 2;
+      ridx[0] = head * dm.dh + jj; ridx[1] = ridx[0] + 1; ridx[2] = ridx[0] + half; ridx[3] = ridx[2] + 1;
+    } else {
+      int r = (dm.Hq + dm.Hkv) * dm.dh + (g - rot_groups) * 4;
+      ridx[0] = r; ridx[1] = r + 1; ridx[2] = r + 2; ridx[3] = r + 3;
+    }
+  } else if (ph.kind == PH_GATEUP) {
+    ridx[0] = 2 * g; ridx[1] = 2 * g + 1; ridx[2] = 2 * g; ridx[3] = 2 * g + 1;
+  } else {
+    ridx[0] = 4 * g; ridx[1] = 4 * g + 1; ridx[2] = 4 * g + 2; ridx[3] = 4 * g + 3;
+  }
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    int r = ridx[j] < ph.R ? ridx[j] : ph.R - 1;
+    const bf16 *base = (ph.kind == PH_GATEUP && j >= 2) ? ph.W2 : ph.W;
+    rows[j] = base + (size_t)r * ph.K;
+  }
+}
+
+// ---- attention work split ----------------------------------------------------
+// Streams: (kv head, group of GQ query heads).  A stream's positions 0..pos are
+// cut into chunks of CH positions (8 KB of K); the last chunk holds the current
+// position and is read with plain loads after the grid barrier, the others go
+// through the ring.  Units u = stream * nch + chunk are dealt to CTAs in
+// contiguous ranges.
+struct AttSplit {
+  int CH, nch, streams, units, u0, u1, gq;
+};
+
+__device__ __forceinline__ AttSplit make_att(const FusedParams &p, int gq, int cta, int ncta) {
+  AttSplit a;
+  a.gq = gq;
+  a.CH = (kStageBytes / 2) / (p.dm.dh * 2);
+  a.nch = p.pos / a.CH + 1;
+  a.streams = p.dm.Hkv * ((p.dm.Hq / p.dm.Hkv) / gq);
+  a.units = a.streams * a.nch;
+  split_range(a.units, cta, ncta, a.u0, a.u1);
+  return a;
+}
+
+__device__ __forceinline__ int cta_of_unit(int u, int units, int ncta) {
+  int c = (int)(((long long)u * ncta) / units);
+  if (c >= ncta) c = ncta - 1;
+  while (c + 1 < ncta && (int)(((long long)units * (c + 1)) / ncta) <= u) ++c;
+  while (c > 0 && (int)(((long long)units * c) / ncta) > u) --c;
+  return c;
+}
+
+// ---- producer ----------------------------------------------------------------
+struct Producer {
+  const Ctx &c;
+  uint32_t s;   // stages issued so far
+  bool ok;
+  __device__ Producer(const Ctx &cc) : c(cc), s(0), ok(true) {}
+  __device__ __forceinline__ bool acquire(uint32_t &slot) {
+    const uint32_t ns = (uint32_t)c.p->n_stages;
+    slot = s % ns;
+    if (s >= ns) {
+      if (!wait_bar(c, smem_u32(&c.empty[slot]), ((s / ns) - 1u) & 1u)) { ok = false; return false; }
+    }
+    return true;
+  }
+  __device__ void gemv_phase(const Phase &ph) {
+    const Dims &dm = c.p->dm;
+    for (int g = ph.g0; g < ph.g1 && ok; ++g) {
+      const bf16 *rows[4];
+      int ridx[4];
+      group_rows(ph, dm, g, rows, ridx);
+      for (int kc = 0; kc < ph.nkc; ++kc) {
+        uint32_t slot;
+        if (!acquire(slot)) return;
+        const int kw = min(kChunk, ph.K - kc * kChunk);
+        const uint32_t bar = smem_u32(&c.full[slot]);
+        const uint32_t dst = smem_u32(c.ring + (size_t)slot * kStageBytes);
+        mbar_expect_tx(bar, 4u * (uint32_t)kw * 2u);
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+          bulk_g2s(dst + j * (kChunk * 2), rows[j] + (size_t)kc * kChunk, (uint32_t)kw * 2u, bar);
+        ++s;
+      }
+    }
+  }
+  __device__ void att_phase(const AttSplit &a, int layer) {
+    const FusedParams &p = *c.p;
+    const Dims &dm = p.dm;
+    const int G = dm.Hq / dm.Hkv, qgroups = G / a.gq;
+    for (int u = a.u0; u < a.u1 && ok; ++u) {
+      const int stream = u / a.nch, chunk = u % a.nch;
+      if (chunk == a.nch - 1) continue;   // the chunk with the current position: plain loads
+      const int kvh = stream / qgroups;
+      uint32_t slot;
+      if (!acquire(slot)) return;
+      const size_t off = ((((size_t)layer * dm.max_slots + p.slot) * dm.Hkv + kvh) * dm.max_seq +
+                          (size_t)chunk * a.CH) * dm.dh;
+      const uint32_t bar = smem_u32(&c.full[slot]);
+      const uint32_t dst = smem_u32(c.ring + (size_t)slot * kStageBytes);
+      mbar_expect_tx(bar, (uint32_t)kStageBytes);
+      bulk_g2s(dst, p.Kc + off, kStageBytes / 2, bar);
+      bulk_g2s(dst + kStageBytes / 2, p.Vc + off, kStageBytes / 2, bar);
+      ++s;
+    }
+  }
+};
+
+// ---- consumer helpers ----------------------------------------------------------
+__device__ __forceinline__ float block_sum(const Ctx &c, float v) {
+  __shared__ float s_part[8];
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  consumer_sync();
+  if ((threadIdx.x & 31) == 0) s_part[threadIdx.x >> 5] = v;
+  consumer_sync();
+  float t = 0.f;
+#pragma unroll
+  for (int w = 0; w < 8; ++w) t += s_part[w];
+  return t;
+}
+
+// position of element k of an activation vector in the permuted shared layout
+__device__ __forceinline__ int act_index(int k) {
+  int kc = k / kChunk, e = k % kChunk;
+  return kc * kChunk + ((e & 7) >> 2) * 1024 + (e >> 3) * 4 + (e & 3);
+}
+
+// act := src (global fp32, length K), optionally RMS-normalised with `gain`
+__device__ void load_act(const Ctx &c, const float *src, int K, const bf16 *gain) {
+  const int tid = threadIdx.x;
+  float scale = 1.f;
+  if (gain) {
+    float ss = 0.f;
+    for (int k = tid * 4; k < K; k += kConsumers * 4) {
+      float4 v = ldcg4(src + k);
+      ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+    }
+    scale = rsqrtf(block_sum(c, ss) / (float)K + c.p->eps);
+  }
+  for (int k = tid * 4; k < K; k += kConsumers * 4) {
+    float4 v = ldcg4(src + k);
+    if (gain) {
+      uint2 gw = *reinterpret_cast<const uint2 *>(gain + k);
+      v.x *= scale * bfl(gw.x); v.y *= scale * bfh(gw.x);
+      v.z *= scale * bfl(gw.y); v.w *= scale * bfh(gw.y);
+    }
+    *reinterpret_cast<float4 *>(c.act + act_index(k)) = v;
+  }
+  consumer_sync();
+}
+
+struct Consumer {
+  const Ctx &c;
+  uint32_t s;     // stages consumed so far
+  uint32_t rbuf;  // parity of the reduction buffer
+  bool ok;
+  __device__ Consumer(const Ctx &cc) : c(cc), s(0), rbuf(0), ok(true) {}
+
+  __device__ __forceinline__ bool wait_stage(uint32_t &slot) {
+    const uint32_t ns = (uint32_t)c.p->n_stages;
+    slot = s % ns;
+    // in abort mode the wait returns at once and the (meaningless) work goes on, so
+    // that every thread still reaches every barrier and the kernel ends
+    if (!wait_bar(c, smem_u32(&c.full[slot]), (s / ns) & 1u)) ok = false;
+    return true;
+  }
+  __device__ __forceinline__ void release_stage(uint32_t slot) {
+    __syncwarp();
+    if ((threadIdx.x & 31) == 0) mbar_arrive(smem_u32(&c.empty[slot]));
+    ++s;
+  }
+
+  // One GEMV phase over the activation vector held in c.act.
+  __device__ void gemv_phase(const Phase &ph, int layer) {
+    const FusedParams &p = *c.p;
+    const Dims &dm = p.dm;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    for (int g = ph.g0; g < ph.g1; ++g) {
+      float acc[4] = {0.f, 0.f, 0.f, 0.f};
+      for (int kc = 0; kc < ph.nkc; ++kc) {
+        uint32_t slot;
+        wait_stage(slot);
+        const int kw = min(kChunk, ph.K - kc * kChunk);
+        if (tid * 8 < kw) {
+          const unsigned char *st = c.ring + (size_t)slot * kStageBytes + tid * 16;
+          const float *a = c.act + kc * kChunk + tid * 4;
+          const float4 x0 = *reinterpret_cast<const float4 *>(a);
+          const float4 x1 = *reinterpret_cast<const float4 *>(a + 1024);
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const uint4 w = *reinterpret_cast<const uint4 *>(st + j * (kChunk * 2));
+            acc[j] += bfl(w.x) * x0.x + bfh(w.x) * x0.y + bfl(w.y) * x0.z + bfh(w.y) * x0.w +
+                      bfl(w.z) * x1.x + bfh(w.z) * x1.y + bfl(w.w) * x1.z + bfh(w.w) * x1.w;
+          }
+        }
+        release_stage(slot);
+      }
+      // block reduction of the four sums, then the epilogue of the group
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) acc[j] += __shfl_xor_sync(0xffffffffu, acc[j], o);
+      }
+      if (lane == 0) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) c.red[rbuf][warp][j] = acc[j];
+      }
+      consumer_sync();
+      if (warp == 0) {
+        float y = 0.f;
+        if (lane < 4) {
+#pragma unroll
+          for (int w = 0; w < 8; ++w) y += c.red[rbuf][w][lane];
+        }
+        const float y0 = __shfl_sync(0xffffffffu, y, 0), y1 = __shfl_sync(0xffffffffu, y, 1);
+        const float y2 = __shfl_sync(0xffffffffu, y, 2), y3 = __shfl_sync(0xffffffffu, y, 3);
+        if (lane == 0) epilogue(ph, dm, layer, g, y0, y1, y2, y3);
+      }
+      rbuf ^= 1u;
+    }
+  }
+
+  __device__ void epilogue(const Phase &ph, const Dims &dm, int layer, int g, float y0, float y1, float y2,
+                           float y3) {
+    const FusedParams &p = *c.p;
+    if (ph.kind == PH_QKV) {
+      const int per_head = dm.dh / 4, half = dm.dh / 2;
+      const int rot_groups = (dm.Hq + dm.Hkv) * per_head;
+      const size_t cbase = ((size_t)layer * dm.max_slots + p.slot) * dm.Hkv;
+      if (g < rot_groups) {
+        const int head = g / per_head, jj = (g % per_head) * 2;
+        const float2 cs0 = p.rope[(size_t)p.pos * half + jj], cs1 = p.rope[(size_t)p.pos * half + jj + 1];
+        const float a0 = y0 * cs0.x - y2 * cs0.y, b0 = y0 * cs0.y + y2 * cs0.x;
+        const float a1 = y1 * cs1.x - y3 * cs1.y, b1 = y1 * cs1.y + y3 * cs1.x;
+        if (head < dm.Hq) {
+          float *q = p.qkv + head * dm.dh;
+          q[jj] = a0; q[jj + 1] = a1; q[jj + half] = b0; q[jj + half + 1] = b1;
+        } else {
+          bf16 *dst = p.Kc + ((cbase + (head - dm.Hq)) * dm.max_seq + p.pos) * dm.dh;
+          dst[jj] = __float2bfloat16_rn(a0); dst[jj + 1] = __float2bfloat16_rn(a1);
+          dst[jj + half] = __float2bfloat16_rn(b0); dst[jj + half + 1] = __float2bfloat16_rn(b1);
+        }
+      } else {
+        const int r = (g - rot_groups) * 4, h = r / dm.dh, e = r % dm.dh;
+        bf16 *dst = p.Vc + ((cbase + h) * dm.max_seq + p.pos) * dm.dh + e;
+        dst[0] = __float2bfloat16_rn(y0); dst[1] = __float2bfloat16_rn(y1);
+        dst[2] = __float2bfloat16_rn(y2); dst[3] = __float2bfloat16_rn(y3);
+      }
+    } else if (ph.kind == PH_GATEUP) {
+      p.u[2 * g] = y0 / (1.f + __expf(-y0)) * y2;
+      p.u[2 * g + 1] = y1 / (1.f + __expf(-y1)) * y3;
+    } else if (ph.kind == PH_HEAD) {
+      const int r = 4 * g;
+      if (r < ph.R) p.logits[r] = y0;
+      if (r + 1 < ph.R) p.logits[r + 1] = y1;
+      if (r + 2 < ph.R) p.logits[r + 2] = y2;
+      if (r + 3 < ph.R) p.logits[r + 3] = y3;
+    } else {   // O-proj / down: residual add on the rows this CTA owns
+      float4 *xp = reinterpret_cast<float4 *>(p.x + 4 * g);
+      float4 v = __ldcg(xp);
+      v.x += y0; v.y += y1; v.z += y2; v.w += y3;
+      *xp = v;
+    }
+  }
+
+  // Attention of this CTA's units; writes one partial (max, sum, o) per stream
+  // segment: part[(stream * ncta + cta)][gq][dh + 2].
+  template <int DH, int GQ>
+  __device__ void att_phase(const AttSplit &a, int layer) {
+    const FusedParams &p = *c.p;
+    const Dims &dm = p.dm;
+    constexpr int EPL = DH / 8;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, part = lane & 7;
+    const int worker = warp * 4 + (lane >> 3);
+    const unsigned wmask = 0xffu << (lane & 24);
+    const int G = dm.Hq / dm.Hkv, qgroups = G / GQ;
+    const float scale = rsqrtf((float)DH);
+    int u = a.u0;
+    while (u < a.u1) {
+      const int stream = u / a.nch;
+      const int kvh = stream / qgroups, qg = stream % qgroups;
+      const int h0 = kvh * G + qg * GQ;
+      const int u_end = min(a.u1, (stream + 1) * a.nch);
+      float q[GQ][EPL], mx[GQ], sum[GQ], o[GQ][EPL];
+#pragma unroll
+      for (int g = 0; g < GQ; ++g) {
+        mx[g] = -INFINITY; sum[g] = 0.f;
+#pragma unroll
+        for (int e = 0; e < EPL; ++e) {
+          q[g][e] = __ldcg(p.qkv + (h0 + g) * DH + part * EPL + e) * scale;
+          o[g][e] = 0.f;
+        }
+      }
+      for (; u < u_end; ++u) {
+        const int chunk = u % a.nch;
+        const bool tail = chunk == a.nch - 1;
+        uint32_t slot = 0;
+        if (!tail) wait_stage(slot);
+        const int t0 = chunk * a.CH;
+        const int cnt = tail ? (p.pos - t0 + 1) : a.CH;
+        const size_t goff = ((((size_t)layer * dm.max_slots + p.slot) * dm.Hkv + kvh) * dm.max_seq + t0) * DH;
+        for (int i = worker; i < cnt; i += 32) {
+          float kf[EPL], vf[EPL];
+          if (tail) {
+            const bf16 *kp = p.Kc + goff + (size_t)i * DH + part * EPL;
+            const bf16 *vp = p.Vc + goff + (size_t)i * DH + part * EPL;
+#pragma unroll
+            for (int e = 0; e < EPL; e += 4) {
+              uint2 kw = __ldcg(reinterpret_cast<const uint2 *>(kp + e));
+              uint2 vw = __ldcg(reinterpret_cast<const uint2 *>(vp + e));
+              kf[e] = bfl(kw.x); kf[e + 1] = bfh(kw.x); kf[e + 2] = bfl(kw.y); kf[e + 3] = bfh(kw.y);
+              vf[e] = bfl(vw.x); vf[e + 1] = bfh(vw.x); vf[e + 2] = bfl(vw.y); vf[e + 3] = bfh(vw.y);
+            }
+          } else {
+            const unsigned char *ks = c.ring + (size_t)slot * kStageBytes + ((size_t)i * DH + part * EPL) * 2;
+            const unsigned char *vs = ks + kStageBytes / 2;
+#pragma unroll
+            for (int e = 0; e < EPL; e += 4) {
+              uint2 kw = *reinterpret_cast<const uint2 *>(ks + e * 2);
+              uint2 vw = *reinterpret_cast<const uint2 *>(vs + e * 2);
+              kf[e] = bfl(kw.x); kf[e + 1] = bfh(kw.x); kf[e + 2] = bfl(kw.y); kf[e + 3] = bfh(kw.y);
+              vf[e] = bfl(vw.x); vf[e + 1] = bfh(vw.x); vf[e + 2] = bfl(vw.y); vf[e + 3] = bfh(vw.y);
+            }
+          }
+#pragma unroll
+          for (int g = 0; g < GQ; ++g) {
+            float sc = 0.f;
+#pragma unroll
+            for (int e = 0; e < EPL; ++e) sc += q[g][e] * kf[e];
+            sc += __shfl_xor_sync(wmask, sc, 1);
+            sc += __shfl_xor_sync(wmask, sc, 2);
+            sc += __shfl_xor_sync(wmask, sc, 4);
+            const float mn = fmaxf(mx[g], sc);
+            const float corr = __expf(mx[g] - mn), pr = __expf(sc - mn);
+            mx[g] = mn;
+            sum[g] = sum[g] * corr + pr;
+#pragma unroll
+            for (int e = 0; e < EPL; ++e) o[g][e] = o[g][e] * corr + pr * vf[e];
+          }
+        }
+        if (!tail) release_stage(slot);
+      }
+      // merge the 32 workers: 4 per warp by shuffles, 8 warps through shared memory
+#pragma unroll
+      for (int off = 8; off <= 16; off <<= 1) {
+#pragma unroll
+        for (int g = 0; g < GQ; ++g) {
+          const float m2 = __shfl_xor_sync(0xffffffffu, mx[g], off);
+          const float s2 = __shfl_xor_sync(0xffffffffu, sum[g], off);
+          const float mn = fmaxf(mx[g], m2);
+          const float c1 = (mx[g] == -INFINITY) ? 0.f : __expf(mx[g] - mn);
+          const float c2 = (m2 == -INFINITY) ? 0.f : __expf(m2 - mn);
+          sum[g] = sum[g] * c1 + s2 * c2;
+#pragma unroll
+          for (int e = 0; e < EPL; ++e) {
+            const float o2 = __shfl_xor_sync(0xffffffffu, o[g][e], off);
+            o[g][e] = o[g][e] * c1 + o2 * c2;
+          }
+          mx[g] = mn;
+        }
+      }
+      float *s_o = c.act;                       // [8][GQ][DH]
+      float *s_ml = c.act + 8 * GQ * DH;        // [8][GQ][2]
+      consumer_sync();                          // the activation buffer is free during attention
+      if (lane < 8) {
+#pragma unroll
+        for (int g = 0; g < GQ; ++g) {
+#pragma unroll
+          for (int e = 0; e < EPL; ++e) s_o[(warp * GQ + g) * DH + part * EPL + e] = o[g][e];
+          if (lane == 0) { s_ml[(warp * GQ + g) * 2] = mx[g]; s_ml[(warp * GQ + g) * 2 + 1] = sum[g]; }
+        }
+      }
+      consumer_sync();
+      float *dst = p.part + ((size_t)stream * c.ncta + c.cta) * (GQ * (DH + 2));
+      for (int i = tid; i < GQ * DH; i += kConsumers) {
+        const int g = i / DH, e = i % DH;
+        float M = -INFINITY;
+#pragma unroll
+        for (int w = 0; w < 8; ++w) M = fmaxf(M, s_ml[(w * GQ + g) * 2]);
+        float Ls = 0.f, O = 0.f;
+#pragma unroll
+        for (int w = 0; w < 8; ++w) {
+          const float mw = s_ml[(w * GQ + g) * 2];
+          const float cf = (mw == -INFINITY) ? 0.f : __expf(mw - M);
+          Ls += s_ml[(w * GQ + g) * 2 + 1] * cf;
+          O += s_o[(w * GQ + g) * DH + e] * cf;
+        }
+        dst[g * (DH + 2) + e] = O;
+        if (e == 0) { dst[g * (DH + 2) + DH] = M; dst[g * (DH + 2) + DH + 1] = Ls; }
+      }
+      consumer_sync();
+    }
+  }
+
+  // act := attention output of all heads, merged from the partials of all CTAs
+  template <int DH, int GQ>
+  __device__ void combine_to_act(const AttSplit &a) {
+    const FusedParams &p = *c.p;
+    const Dims &dm = p.dm;
+    const int G = dm.Hq / dm.Hkv, qgroups = G / GQ;
+    for (int i = threadIdx.x; i < dm.Hq * DH; i += kConsumers) {
+      const int h = i / DH, e = i % DH;
+      const int kvh = h / G, qg = (h % G) / GQ, g = (h % G) % GQ;
+      const int stream = kvh * qgroups + qg;
+      const int c0 = cta_of_unit(stream * a.nch, a.units, c.ncta);
+      const int c1 = cta_of_unit((stream + 1) * a.nch - 1, a.units, c.ncta);
+      // CTAs c0..c1 hold the stream's units; one with an empty range wrote nothing
+      float M = -INFINITY;
+      for (int cc = c0; cc <= c1; ++cc) {
+        if ((long long)a.units * cc / c.ncta == (long long)a.units * (cc + 1) / c.ncta) continue;
+        M = fmaxf(M, __ldcg(p.part + ((size_t)stream * c.ncta + cc) * (GQ * (DH + 2)) + g * (DH + 2) + DH));
+      }
+      float Ls = 0.f, O = 0.f;
+      for (int cc = c0; cc <= c1; ++cc) {
+        if ((long long)a.units * cc / c.ncta == (long long)a.units * (cc + 1) / c.ncta) continue;
+        const float *src = p.part + ((size_t)stream * c.ncta + cc) * (GQ * (DH + 2)) + g * (DH + 2);
+        const float cf = __expf(__ldcg(src + DH) - M);
+        Ls += __ldcg(src + DH + 1) * cf;
+        O += __ldcg(src + e) * cf;
+      }
+      c.act[act_index(i)] = O / Ls;
+    }
+    consumer_sync();
+  }
+};
+
+template <int DH, int GQ>
+__global__ void __launch_bounds__(kFusedThreads, 1) k_step_b1(const __grid_constant__ FusedParams p) {
+  extern __shared__ __align__(128) unsigned char smem[];
+  __shared__ __align__(8) uint64_t s_full[kMaxStages], s_empty[kMaxStages];
+  __shared__ float s_red[2][8][4];
+  __shared__ int s_abort;
+  const int tid = threadIdx.x, warp = tid >> 5;
+  Ctx c;
+  c.p = &p;
+  c.ring = smem;
+  c.act = reinterpret_cast<float *>(smem + (size_t)p.n_stages * kStageBytes);
+  c.full = s_full; c.empty = s_empty;
+  c.abort_flag = &s_abort;
+  c.red = s_red;
+  c.cta = blockIdx.x; c.ncta = gridDim.x;
+  if (tid == 0) {
+    s_abort = 0;
+    for (int i = 0; i < p.n_stages; ++i) {
+      mbar_init(smem_u32(&s_full[i]), 1);
+      mbar_init(smem_u32(&s_empty[i]), 8);
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  __syncthreads();
+
+  // depth schedule of the row (every thread, integers only):
+  // floor(L alpha^i) = #{ n in 1..L : i < thr[n] }
+  const int L = p.L;
+  int n = 0;
+  for (int k = 1; k <= L; ++k) n += (p.gi < p.thr[k]) ? 1 : 0;
+  int lo, hi;
+  if (p.anchor == D3_ANCHOR_TAIL) { lo = n; hi = L; }
+  else { if (n < p.start_id) n = p.start_id; lo = p.start_id; hi = p.start_id + (L - n); }
+
+  const AttSplit att = make_att(p, GQ, c.cta, c.ncta);
+
+  if (warp == 8) {
+    // ------------------------------------------------------------ producer
+    if ((tid & 31) == 0) {
+      Producer pr(c);
+      for (int l = 0; l < L && pr.ok; ++l) {
+        if (lo <= l && l < hi) continue;
+        pr.gemv_phase(make_phase(p, PH_QKV, l, c.cta, c.ncta));
+        pr.att_phase(att, l);
+        pr.gemv_phase(make_phase(p, PH_OPROJ, l, c.cta, c.ncta));
+        pr.gemv_phase(make_phase(p, PH_GATEUP, l, c.cta, c.ncta));
+        pr.gemv_phase(make_phase(p, PH_DOWN, l, c.cta, c.ncta));
+      }
+      if (pr.ok && p.logits) pr.gemv_phase(make_phase(p, PH_HEAD, 0, c.cta, c.ncta));
+      if (!pr.ok) {
+        // drain: wait (bounded) until every copy already issued has landed
+        const uint32_t ns = (uint32_t)p.n_stages;
+        const uint32_t first = pr.s > ns ? pr.s - ns : 0;
+        for (uint32_t s = first; s < pr.s; ++s) {
+          const uint32_t bar = smem_u32(&s_full[s % ns]);
+          const uint64_t t0 = now_ns();
+          while (!mbar_try_wait(bar, (s / ns) & 1u) && now_ns() - t0 < p.wait_ns) {}
+        }
+      }
+    }
+    return;
+  }
+
+  // -------------------------------------------------------------- consumers
+  const int tok = p.tok_dev ? p.tok_dev[0] : p.tok;
+  if (c.cta == 0 && tid == 0) {
+    DevSched *s = p.sched;
+    s->B = 1; s->L = L; s->n[0] = n; s->perm[0] = 0; s->slot_s[0] = p.slot; s->pos_s[0] = p.pos;
+    s->tok_s[0] = tok; s->lo_s[0] = lo; s->hi_s[0] = hi;
+    for (int l = 0; l < L; ++l) s->m[l] = (lo <= l && l < hi) ? 0 : 1;
+    s->rows_layers = n; s->layers_touched = n;
+  }
+  // embedding row -> residual stream (CTA 0 publishes it; everybody normalises its own copy)
+  const Dims &dm = p.dm;
+  if (c.cta == 0) {
+    const bf16 *e = p.embed + (size_t)tok * dm.d;
+    for (int k = tid * 8; k < dm.d; k += kConsumers * 8) {
+      uint4 w = *reinterpret_cast<const uint4 *>(e + k);
+      *reinterpret_cast<float4 *>(p.x + k) = make_float4(bfl(w.x), bfh(w.x), bfl(w.y), bfh(w.y));
+      *reinterpret_cast<float4 *>(p.x + k + 4) = make_float4(bfl(w.z), bfh(w.z), bfl(w.w), bfh(w.w));
+    }
+  }
+  Consumer cs(c);
+  unsigned bidx = 0;
+  grid_barrier(c, ++bidx);
+  for (int l = 0; l < L; ++l) {
+    if (lo <= l && l < hi) continue;   // dropped block: the hidden state passes through
+    load_act(c, p.x, dm.d, p.layers[l].attn_norm);
+    cs.gemv_phase(make_phase(p, PH_QKV, l, c.cta, c.ncta), l);
+    grid_barrier(c, ++bidx);
+    cs.template att_phase<DH, GQ>(att, l);
+    grid_barrier(c, ++bidx);
+    cs.template combine_to_act<DH, GQ>(att);
+    cs.gemv_phase(make_phase(p, PH_OPROJ, l, c.cta, c.ncta), l);
+    grid_barrier(c, ++bidx);
+    load_act(c, p.x, dm.d, p.layers[l].mlp_norm);
+    cs.gemv_phase(make_phase(p, PH_GATEUP, l, c.cta, c.ncta), l);
+    grid_barrier(c, ++bidx);
+    load_act(c, p.u, dm.f, nullptr);
+    cs.gemv_phase(make_phase(p, PH_DOWN, l, c.cta, c.ncta), l);
+    grid_barrier(c, ++bidx);
+  }
+  // KV fill by copy for the dropped blocks: CTA j takes block lo + j, lo + j + ncta, ...
+  if (p.kv_fill == D3_FILL_COPY) {
+    const int nkv = dm.Hkv * dm.dh;
+    for (int l = lo + c.cta; l < hi; l += c.ncta) {
+      for (int i = tid; i < nkv; i += kConsumers) {
+        const int h = i / dm.dh, e = i % dm.dh;
+        const size_t dst = ((((size_t)l * dm.max_slots + p.slot) * dm.Hkv + h) * dm.max_seq + p.pos) * dm.dh + e;
+        if (lo == 0) {
+          p.Kc[dst] = __float2bfloat16_rn(0.f);
+          p.Vc[dst] = __float2bfloat16_rn(0.f);
+        } else {
+          const size_t src = ((((size_t)(lo - 1) * dm.max_slots + p.slot) * dm.Hkv + h) * dm.max_seq + p.pos) * dm.dh + e;
+          unsigned short *Ku = reinterpret_cast<unsigned short *>(p.Kc);
+          unsigned short *Vu = reinterpret_cast<unsigned short *>(p.Vc);
+          Ku[dst] = __ldcg(Ku + src);   // written by another CTA earlier in this kernel
+          Vu[dst] = __ldcg(Vu + src);
+        }
+      }
+    }
+  }
+  if (p.logits) {
+    load_act(c, p.x, dm.d, p.final_norm);
+    cs.gemv_phase(make_phase(p, PH_HEAD, 0, c.cta, c.ncta), 0);
+  }
+}
+
+}  // namespace
+
+// ------------------------------------------------------------------ host side
+struct FusedPlan {
+  int ok;            // 1 when the fused kernel serves this model
+  int grid, n_stages, act_floats;
+  size_t smem;
+  void *func;
+};
+
+template <int DH, int GQ>
+static bool try_plan(FusedPlan &pl, const d3_config &c) {
+  int dev = 0, sms = 0, optin = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return false;
+  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+  int coop = 0;
+  cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev);
+  if (!coop || sms < 1) return false;
+  int need = c.d_model;
+  if (c.d_ffn > need) need = c.d_ffn;
+  if (c.n_q_heads * c.head_dim > need) need = c.n_q_heads * c.head_dim;
+  need = (need + kChunk - 1) / kChunk * kChunk;
+  const int att_need = 8 * kMaxGQ * (128 + 2);
+  if (need < att_need) need = (att_need + kChunk - 1) / kChunk * kChunk;
+  const int reserve = 4096;   // static shared memory of the kernel and slack
+  int stages = (optin - reserve - need * 4) / kStageBytes;
+  if (stages > kMaxStages) stages = kMaxStages;
+  if (stages < 3) return false;
+  pl.n_stages = stages;
+  pl.act_floats = need;
+  pl.smem = (size_t)stages * kStageBytes + (size_t)need * 4;
+  pl.func = (void *)k_step_b1<DH, GQ>;
+  if (cudaFuncSetAttribute(k_step_b1<DH, GQ>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem) !=
+      cudaSuccess)
+    return false;
+  int per_sm = 0;
+  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_step_b1<DH, GQ>, kFusedThreads, pl.smem) !=
+          cudaSuccess ||
+      per_sm < 1)
+    return false;
+  pl.grid = sms;
+  pl.ok = 1;
+  return true;
+}
+
+int fused_plan(const d3_config &c, int *grid, int *n_stages, int *act_floats, size_t *smem, void **func) {
+  FusedPlan pl;
+  memset(&pl, 0, sizeof(pl));
+  const int G = c.n_q_heads / c.n_kv_heads;
+  const int gq = (G % 4 == 0) ? 4 : (G % 2 == 0) ? 2 : 1;
+  bool ok = false;
+  if (c.vocab % 4 == 0 && c.head_dim * 2 * c.max_seq % 16 == 0) {
+    if (c.head_dim == 128 && gq == 1) ok = try_plan<128, 1>(pl, c);
+    else if (c.head_dim == 128 && gq == 4) ok = try_plan<128, 4>(pl, c);
+    else if (c.head_dim == 64 && gq == 1) ok = try_plan<64, 1>(pl, c);
+    else if (c.head_dim == 32 && gq == 4) ok = try_plan<32, 4>(pl, c);
+  }
+  cudaGetLastError();   // a failed attribute call must not poison later launches
+  if (!ok) return 0;
+  *grid = pl.grid; *n_stages = pl.n_stages; *act_floats = pl.act_floats; *smem = pl.smem; *func = pl.func;
+  return 1;
+}
+
+int launch_fused_step(void *func, int grid, size_t smem, FusedParams &fp, cudaStream_t st) {
+  if (cudaMemsetAsync(fp.bar_counter, 0, sizeof(unsigned), st) != cudaSuccess) return -1;
+  void *args[] = {(void *)&fp};
+  if (cudaLaunchCooperativeKernel(func, dim3(grid), dim3(kFusedThreads), args, smem, st) != cudaSuccess)
+    return -1;
+  return 1;
+}
+
+}  // namespace d3

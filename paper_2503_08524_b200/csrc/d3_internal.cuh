@@ -72,9 +72,36 @@ struct Dims {
   int L, d, Hq, Hkv, dh, f, V, max_slots, max_seq, qkv_rows;
 };
 
+// device table of one block's weight pointers (fused step kernel)
+struct LayerPtrs {
+  const bf16 *attn_norm, *wqkv, *wo, *mlp_norm, *w_gate, *w_up, *w_down;
+};
+
+static constexpr int kFusedMaxCtas = 192;
+
+// parameters of the fused batch-1 step kernel (passed by value)
+struct FusedParams {
+  int32_t slot, tok, gi, pos;
+  const int32_t *tok_dev;
+  int32_t thr[D3_MAX_LAYERS + 1];
+  int32_t L, start_id, anchor, kv_fill;
+  Dims dm;
+  float eps;
+  const LayerPtrs *layers;
+  const bf16 *embed, *lm_head, *final_norm;
+  bf16 *Kc, *Vc;
+  const float2 *rope;
+  DevSched *sched;
+  unsigned *bar_counter;
+  float *x, *qkv, *u, *part;
+  float *logits;
+  int32_t n_stages, act_floats;
+  unsigned long long wait_ns;   // bound of every device-side wait
+};
+
 // Byte offsets of the regions of the caller's scratch buffer.
 struct Layout {
-  size_t sched, rope, x, qkv, attn_out, part_o, part_ml, u, total;
+  size_t sched, rope, x, qkv, attn_out, part_o, part_ml, u, layer_tab, bar, part_fused, total;
   int max_splits;
 };
 
@@ -94,5 +121,8 @@ int launch_attention(const float *qkv, const bf16 *Kc, const bf16 *Vc, const Dev
 int launch_fill_copy(bf16 *Kc, bf16 *Vc, const DevSched *s, int B, const Dims &dm, cudaStream_t st);
 int launch_argmax(const float *logits, int B, int V, int32_t *out, cudaStream_t st);
 int init_kernel_attributes();
+// fused batch-1 step: returns 1 and the launch plan when the kernel serves `c` on this device
+int fused_plan(const d3_config &c, int *grid, int *n_stages, int *act_floats, size_t *smem, void **func);
+int launch_fused_step(void *func, int grid, size_t smem, FusedParams &fp, cudaStream_t st);
 
 }  // namespace d3

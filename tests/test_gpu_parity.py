@@ -71,8 +71,10 @@ def test_schedule_kernel_large_L(B):
 @pytest.mark.parametrize("shape", [I.TINY, I.TINY_GQA], ids=["mha", "gqa"])
 @pytest.mark.parametrize("alpha", [1.0, 0.98, 0.95])
 @pytest.mark.parametrize("kv_round", [False, True], ids=["kv-exact", "kv-bf16"])
-def test_tiny_generate_teacher_forced(B, shape, alpha, kv_round):
+@pytest.mark.parametrize("exec_mode", [0, 1], ids=["fused", "kernels"])
+def test_tiny_generate_teacher_forced(B, shape, alpha, kv_round, exec_mode):
     orc, gpu = make_pair(shape, SEED, 2, 64, 1, start_id=0, kv_round_bf16=kv_round)
+    gpu.d3_set_exec(exec_mode)
     prompt = I.prompt_tokens(shape, SEED, 0, 16).numpy()
     o_lg, o_hid = orc.prefill(1, prompt, want_hidden=True)
     g_lg = gpu.d3_prefill(1, prompt)
@@ -160,6 +162,41 @@ def test_batched_mixed_depth_steps(B, anchor, start, fill):
     gpu.close()
 
 
+@pytest.mark.parametrize("anchor,start", [(0, 0), (0, 1), (0, 3), (1, 0)])
+@pytest.mark.parametrize("fill", [0, 1])
+def test_fused_step_fills_and_long_context(B, anchor, start, fill):
+    # batch 1 through the single-kernel step: several KV chunks per head (the
+    # last one ragged), windows at both anchors, cache contents against the oracle
+    shape = I.TINY_GQA
+    orc, gpu = make_pair(shape, SEED + 7, 1, 700, 16, start_id=start, anchor=anchor, kv_fill=fill)
+    gpu.poison_kv()
+    orc.poison_kv()
+    prompt = I.prompt_tokens(shape, SEED + 7, 0, 389).numpy()
+    o = orc.prefill(0, prompt)
+    g = gpu.d3_prefill(0, prompt)
+    check_step("prefill", g.cpu().numpy()[None], None, o[None], None)
+    toks = I.token_ids(SEED + 7, 5, 40, shape.vocab).numpy()
+    for i in range(1, 30):
+        r = orc.decode_step([0], [int(toks[i])], [i], 0.93)
+        g, st = gpu.d3_decode_step([0], [int(toks[i])], [i], 0.93, want_stats=True)
+        assert st["kernel_launches"] == 1
+        check_step(f"step {i}", g.cpu().numpy(), gpu.d3_read_hidden(1), r["logits"], r["hidden"])
+        dev = gpu.d3_read_schedule(1)
+        want = O.schedule(shape.n_layers, 0.93, start, anchor, [i])
+        assert np.array_equal(dev["n"], want["n"]) and np.array_equal(dev["m_per_layer"], want["m_per_layer"])
+        pos = orc.slot_pos(0) - 1
+        for l in range(shape.n_layers):
+            ok, ov = orc.read_kv(l, 0, pos)
+            gk, gv = gpu.d3_read_kv(l, 0, pos)
+            if np.isnan(ok).any():
+                assert np.isnan(gk).all() and np.isnan(gv).all()
+            else:
+                assert np.abs(gk - ok).max() <= 0.02 * max(1.0, np.abs(ok).max())
+                assert np.abs(gv - ov).max() <= 0.02 * max(1.0, np.abs(ov).max())
+    gpu.d3_sync()
+    gpu.close()
+
+
 @pytest.mark.parametrize("fill", [1, 2])
 def test_alpha_raised_mid_sequence_reads_filled_entries(B, fill):
     # depth grows again when the caller raises alpha: later tokens then read what
@@ -198,8 +235,10 @@ def test_prefill_longer_than_a_batch_and_ragged_lengths(B):
 
 # ----------------------------------------------------------- production widths
 
-@pytest.mark.parametrize("base,layers,Bn", [(I.LLAMA_7B, 3, 1), (I.LLAMA_7B, 2, 5), (I.LLAMA_70B, 2, 3)],
-                         ids=["7b-width-b1", "7b-width-b5", "70b-width-gqa-b3"])
+@pytest.mark.parametrize("base,layers,Bn", [(I.LLAMA_7B, 3, 1), (I.LLAMA_7B, 2, 5), (I.LLAMA_70B, 2, 3),
+                                            (I.LLAMA_13B, 2, 1), (I.LLAMA_70B, 2, 1)],
+                         ids=["7b-width-b1", "7b-width-b5", "70b-width-gqa-b3", "13b-width-b1",
+                              "70b-width-gqa-b1"])
 def test_production_widths(B, base, layers, Bn):
     # full-width blocks (same kernel shapes and tiling as the benchmark), few layers
     shape = base.with_layers(layers)
