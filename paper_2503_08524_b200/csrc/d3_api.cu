@@ -28,7 +28,8 @@ Layout make_layout(const d3_config &c) {
   y.part_ml = off;  off = align_up(off + B * c.n_q_heads * y.max_splits * 2 * 4, 256);
   y.u = off;        off = align_up(off + B * c.d_ffn * 4, 256);
   y.layer_tab = off; off = align_up(off + (size_t)c.n_layers * sizeof(LayerPtrs), 256);
-  y.bar = off;      off = align_up(off + 256, 256);
+  y.bar = off;      off = align_up(off + kFusedSyncBytes, 256);
+  y.phase = off;    off = align_up(off + (size_t)kFusedMaxCtas * kFusedPhases * 8, 256);
   y.part_fused = off;
   off = align_up(off + (size_t)c.n_q_heads * kFusedMaxCtas * (c.head_dim + 2) * 4, 256);
   y.total = off;
@@ -96,8 +97,8 @@ struct d3_model {
   bool prof_on;
   std::vector<cudaEvent_t> prof_events;   // pool, two per recorded launch
   std::vector<int> prof_kind;             // kind of each recorded pair of the running step
-  float prof_ms[D3_PROF_KINDS];
-  int32_t prof_n[D3_PROF_KINDS];
+  float prof_ms[10];
+  int32_t prof_n[10];
   // fused batch-1 step kernel
   int32_t exec_mode;
   int fused_ok, fused_grid, fused_stages, fused_act;
@@ -117,9 +118,14 @@ struct d3_model {
 
 enum ProfKind { PK_SCHED = 0, PK_QKV, PK_ROPE, PK_ATTN, PK_OPROJ, PK_GATEUP, PK_DOWN, PK_FILL,
                 PK_HEAD, PK_FUSED };
-static const char *kProfNames[D3_PROF_KINDS] = {"schedule+embed", "norm+qkv", "rope+kv_append",
-                                                "attention", "o_proj+resid", "norm+gate_up+swiglu",
-                                                "down+resid", "kv_fill", "norm+lm_head", "fused_step"};
+static const char *kProfNames[D3_PROF_KINDS] = {
+    "schedule+embed", "norm+qkv", "rope+kv_append", "attention", "o_proj+resid", "norm+gate_up+swiglu",
+    "down+resid", "kv_fill", "norm+lm_head", "fused_step",
+    // phases inside the fused step kernel (mean over CTAs, nominal-clock ms)
+    "fused:prologue", "fused:load_act", "fused:qkv", "fused:grid_barriers", "fused:attention",
+    "fused:o_proj", "fused:gate_up", "fused:down", "fused:head+fill",
+    // smallest and largest per-CTA time spent in grid barriers
+    "fused:grid_barriers_min", "fused:grid_barriers_max"};
 
 // Scope that brackets one launch (or a launcher's pair of launches) with events.
 struct ProfScope {
@@ -273,7 +279,9 @@ static int32_t run_fused_step(d3_model *m, const StepArgs &a, float *logits_dev,
   fp.embed = m->embed; fp.lm_head = m->lm_head; fp.final_norm = m->final_norm;
   fp.Kc = m->Kc; fp.Vc = m->Vc; fp.rope = m->rope(); fp.sched = m->sched();
   fp.bar_counter = reinterpret_cast<unsigned *>(m->scratch + m->lay.bar);
-  fp.x = m->x(); fp.qkv = m->qkv(); fp.u = m->u();
+  fp.stream_count = fp.bar_counter + 16;
+  fp.phase_cycles = m->prof_on ? reinterpret_cast<long long *>(m->scratch + m->lay.phase) : nullptr;
+  fp.x = m->x(); fp.qkv = m->qkv(); fp.u = m->u(); fp.attn_out = m->attn_out();
   fp.part = reinterpret_cast<float *>(m->scratch + m->lay.part_fused);
   fp.logits = logits_dev;
   fp.n_stages = m->fused_stages; fp.act_floats = m->fused_act;
@@ -406,7 +414,12 @@ int32_t d3_load(const d3_config *cfg, const d3_weights *w, void *kv_dev, void *s
   m->fused_ok = fused_plan(*cfg, &m->fused_grid, &m->fused_stages, &m->fused_act, &m->fused_smem,
                            &m->fused_func);
   if (m->fused_ok && m->fused_grid > kFusedMaxCtas) m->fused_grid = kFusedMaxCtas;
-  if (cudaMemsetAsync(m->sched(), 0, sizeof(DevSched), m->stream) != cudaSuccess) { delete m; return D3_ECUDA; }
+  if (cudaMemsetAsync(m->sched(), 0, sizeof(DevSched), m->stream) != cudaSuccess ||
+      cudaMemsetAsync(m->scratch + m->lay.phase, 0, (size_t)kFusedMaxCtas * kFusedPhases * 8, m->stream) !=
+          cudaSuccess) {
+    delete m;
+    return D3_ECUDA;
+  }
   launch_rope_table(m->rope(), cfg->max_seq, cfg->head_dim, cfg->rope_base, m->stream);
   if (cudaGetLastError() != cudaSuccess) { delete m; return D3_ECUDA; }
   *out = m;
@@ -586,8 +599,38 @@ int32_t d3_profile(d3_model *m, int32_t enable) {
 
 int32_t d3_read_profile(d3_model *m, float *ms, int32_t *launches) {
   if (!m || !ms || !launches) return D3_EINVAL;
+  memset(ms, 0, sizeof(float) * D3_PROF_KINDS);
+  memset(launches, 0, sizeof(int32_t) * D3_PROF_KINDS);
   memcpy(ms, m->prof_ms, sizeof(m->prof_ms));
   memcpy(launches, m->prof_n, sizeof(m->prof_n));
+  if (m->fused_ok && m->prof_n[PK_FUSED] > 0) {
+    // phases of the fused step kernel, timed by every CTA in SM cycles
+    std::vector<long long> cyc((size_t)kFusedMaxCtas * kFusedPhases);
+    int dev = 0, khz = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&khz, cudaDevAttrClockRate, dev);
+    if (cudaStreamSynchronize(m->stream) != cudaSuccess) return D3_ECUDA;
+    char *ph = m->scratch + m->lay.phase;
+    if (cudaMemcpy(cyc.data(), ph, cyc.size() * 8, cudaMemcpyDeviceToHost) != cudaSuccess) return D3_ECUDA;
+    if (cudaMemset(ph, 0, cyc.size() * 8) != cudaSuccess) return D3_ECUDA;
+    const double to_ms = khz > 0 ? 1.0 / (double)khz : 0.0;
+    const int nc = m->fused_grid;
+    for (int k = 0; k < kFusedPhases; ++k) {
+      double tot = 0;
+      for (int cta = 0; cta < nc; ++cta) tot += (double)cyc[(size_t)cta * kFusedPhases + k];
+      ms[D3_PROF_FUSED0 + k] = (float)(tot / nc * to_ms);
+      launches[D3_PROF_FUSED0 + k] = m->prof_n[PK_FUSED];
+    }
+    long long mn = cyc[3], mx = cyc[3];
+    for (int cta = 0; cta < nc; ++cta) {
+      const long long v = cyc[(size_t)cta * kFusedPhases + 3];
+      if (v < mn) mn = v;
+      if (v > mx) mx = v;
+    }
+    ms[D3_PROF_FUSED0 + kFusedPhases] = (float)(mn * to_ms);
+    ms[D3_PROF_FUSED0 + kFusedPhases + 1] = (float)(mx * to_ms);
+    launches[D3_PROF_FUSED0 + kFusedPhases] = launches[D3_PROF_FUSED0 + kFusedPhases + 1] = m->prof_n[PK_FUSED];
+  }
   memset(m->prof_ms, 0, sizeof(m->prof_ms));
   memset(m->prof_n, 0, sizeof(m->prof_n));
   return D3_OK;

@@ -1,23 +1,30 @@
 // Batch-1 decode step as ONE persistent cooperative kernel (sm_100a).
 //
-// One CTA per SM.  Warp 8 is the producer: a single thread streams the CTA's
-// share of every weight matrix (and of the static part of the KV cache) through
-// a shared-memory ring with bulk asynchronous copies (cp.async.bulk + mbarrier
+// One CTA per SM.  Warp 8 is the producer: it streams the CTA's share of every
+// weight matrix (and of the static part of the KV cache) through a
+// shared-memory ring with bulk asynchronous copies (cp.async.bulk + mbarrier
 // transaction counts).  It never waits for the computation, so HBM stays busy
-// across phase boundaries: weights do not depend on activations.  Warps 0-7
-// consume ring stages in lockstep.  Phases of a block (RMSNorm+QKV+RoPE+KV
-// append | attention | O-proj+residual | RMSNorm+gate/up+SwiGLU | down+residual)
-// are separated by grid barriers on a global counter; only the small fp32
-// activations cross them (through L2, read with ld.global.cg).
+// across phase boundaries: weights do not depend on activations.  Each ring
+// stage is consumed by ONE of the warps 0-7 (stage s of a phase by warp s mod 8),
+// so the warps work on eight stages at a time and never synchronise inside a
+// projection.  Phases of a block (RMSNorm+QKV+RoPE+KV append | attention |
+// O-proj+residual | RMSNorm+gate/up+SwiGLU | down+residual) are separated by
+// grid barriers on a global counter; only the small fp32 activations cross them
+// (through L2, read with ld.global.cg).
 //
 // A ring stage is 16 KB: four weight-row segments of 2048 bf16 (a "row group" x
-// k-chunk), or 8 KB of K plus 8 KB of V for one KV head.  In a GEMV stage thread
-// t owns k = t*8..t*8+7 of the chunk for all four rows, so the activation costs
-// two shared loads per four weight loads.
+// k-chunk), or 8 KB of K plus 8 KB of V for one KV head.  Row groups are issued
+// eight at a time, k-chunk major, so that warp w keeps the four running sums of
+// group w in registers across the k-chunks and finishes the group alone
+// (shuffle reduction + epilogue).  A lane owns 8 consecutive k of every
+// 256-element block, so the activation costs two shared loads per four weight
+// loads.
 //
-// Every wait (mbarrier, grid barrier) is bounded; on expiry the kernel raises
-// D3_ETIMEOUT in the schedule's status word, stops issuing copies, drains the
-// copies in flight and returns.
+// Every wait (mbarrier, release counter, grid barrier) is bounded in time; on
+// expiry the kernel raises D3_ETIMEOUT in the schedule's status word and enters
+// abort mode: waits return at once, the producer stops issuing and drains the
+// copies in flight, and every thread still walks the same control flow to the
+// end so that no barrier is left waiting.
 #include "d3_internal.cuh"
 
 namespace d3 {
@@ -66,29 +73,26 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void *src, uint32_t
       : "memory");
 }
 __device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
-
 __device__ __forceinline__ float4 ldcg4(const float *p) { return __ldcg(reinterpret_cast<const float4 *>(p)); }
-
-}  // namespace
-
-
-namespace {
+__device__ __forceinline__ uint64_t now_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
 
 struct Ctx {
   const FusedParams *p;
   unsigned char *ring;
   float *act;
   uint64_t *full, *empty;
+  volatile uint32_t *released;   // per slot: fills consumed so far
   volatile int *abort_flag;
-  float (*red)[8][4];
   int cta, ncta;
 };
 
-// ---- bounded waits ---------------------------------------------------------
-__device__ __forceinline__ uint64_t now_ns() {
-  uint64_t t;
-  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-  return t;
+__device__ __forceinline__ void raise_timeout(const Ctx &c) {
+  c.p->sched->status = D3_ETIMEOUT;
+  *c.abort_flag = 1;
 }
 
 // Wait for an mbarrier phase for at most wait_ns.  Returns false at once when
@@ -104,13 +108,12 @@ __device__ __forceinline__ bool wait_bar(const Ctx &c, uint32_t bar, uint32_t pa
       if (now_ns() - t0 > c.p->wait_ns) break;
     }
   }
-  c.p->sched->status = D3_ETIMEOUT;
-  *c.abort_flag = 1;
+  raise_timeout(c);
   return false;
 }
 
 // Grid barrier number `idx` (1-based) among the consumer threads of all CTAs.
-__device__ __forceinline__ bool grid_barrier(const Ctx &c, unsigned idx) {
+__device__ __forceinline__ void grid_barrier(const Ctx &c, unsigned idx) {
   consumer_sync();
   if (threadIdx.x == 0) {
     __threadfence();
@@ -121,15 +124,11 @@ __device__ __forceinline__ bool grid_barrier(const Ctx &c, unsigned idx) {
       unsigned v;
       asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(c.p->bar_counter) : "memory");
       if (v >= target) break;
-      if ((it & 15u) == 0u && now_ns() - t0 > c.p->wait_ns) {
-        c.p->sched->status = D3_ETIMEOUT;
-        *c.abort_flag = 1;
-      }
+      if ((it & 15u) == 0u && now_ns() - t0 > c.p->wait_ns) raise_timeout(c);
     }
     __threadfence();
   }
   consumer_sync();
-  return *c.abort_flag == 0;
 }
 
 // ---- the CTA's share of a phase ---------------------------------------------
@@ -162,29 +161,26 @@ __device__ __forceinline__ Phase make_phase(const FusedParams &p, int kind, int 
   return ph;
 }
 
-// the four weight rows of group g (row pointers; rows beyond R are clamped)
-__device__ __forceinline__ void group_rows(const Phase &ph, const Dims &dm, int g, const bf16 *rows[4], int ridx[4]) {
+// pointer of weight row j (0..3) of group g (rows beyond R are clamped)
+__device__ __forceinline__ const bf16 *group_row(const Phase &ph, const Dims &dm, int g, int j) {
+  int r;
   if (ph.kind == PH_QKV) {
     const int per_head = dm.dh / 4, half = dm.dh / 2;
     const int rot_groups = (dm.Hq + dm.Hkv) * per_head;
-    if (g < rot_groups) {   // q or k head: two rotary pairs (j, j+half), (j+1, j+1+half)
-      int head = g / per_head, jj = (g % per_head) * 2;
-      ridx[0] = head * dm.dh + jj; ridx[1] = ridx[0] + 1; ridx[2] = ridx[0] + half; ridx[3] = ridx[2] + 1;
+    if (g < rot_groups) {   // q or k head: two rotary pairs (jj, jj+half), (jj+1, jj+1+half)
+      const int head = g / per_head, jj = (g % per_head) * 2;
+      r = head * dm.dh + jj + (j & 1) + (j >> 1) * half;
     } else {
-      int r = (dm.Hq + dm.Hkv) * dm.dh + (g - rot_groups) * 4;
-      ridx[0] = r; ridx[1] = r + 1; ridx[2] = r + 2; ridx[3] = r + 3;
+      r = (dm.Hq + dm.Hkv) * dm.dh + (g - rot_groups) * 4 + j;
     }
   } else if (ph.kind == PH_GATEUP) {
-    ridx[0] = 2 * g; ridx[1] = 2 * g + 1; ridx[2] = 2 * g; ridx[3] = 2 * g + 1;
+    r = 2 * g + (j & 1);   // rows 0,1: gate; rows 2,3: up
   } else {
-    ridx[0] = 4 * g; ridx[1] = 4 * g + 1; ridx[2] = 4 * g + 2; ridx[3] = 4 * g + 3;
+    r = 4 * g + j;
   }
-#pragma unroll
-  for (int j = 0; j < 4; ++j) {
-    int r = ridx[j] < ph.R ? ridx[j] : ph.R - 1;
-    const bf16 *base = (ph.kind == PH_GATEUP && j >= 2) ? ph.W2 : ph.W;
-    rows[j] = base + (size_t)r * ph.K;
-  }
+  if (r >= ph.R) r = ph.R - 1;
+  const bf16 *base = (ph.kind == PH_GATEUP && j >= 2) ? ph.W2 : ph.W;
+  return base + (size_t)r * ph.K;
 }
 
 // ---- attention work split ----------------------------------------------------
@@ -216,7 +212,7 @@ __device__ __forceinline__ int cta_of_unit(int u, int units, int ncta) {
   return c;
 }
 
-// ---- producer ----------------------------------------------------------------
+// ---- producer (all 32 lanes of warp 8 run it) -----------------------------------
 struct Producer {
   const Ctx &c;
   uint32_t s;   // stages issued so far
@@ -230,29 +226,34 @@ struct Producer {
     }
     return true;
   }
+  // Lane 4w+j holds the pointer of row j of group w of the current batch of eight
+  // groups; the four lanes of a group issue its copies.
   __device__ void gemv_phase(const Phase &ph) {
     const Dims &dm = c.p->dm;
-    for (int g = ph.g0; g < ph.g1 && ok; ++g) {
-      const bf16 *rows[4];
-      int ridx[4];
-      group_rows(ph, dm, g, rows, ridx);
+    const int lane = threadIdx.x & 31, w = lane >> 2, j = lane & 3;
+    for (int S0 = ph.g0; S0 < ph.g1 && ok; S0 += 8) {
+      const int nw = min(8, ph.g1 - S0);
+      const bf16 *row = (w < nw) ? group_row(ph, dm, S0 + w, j) : nullptr;
       for (int kc = 0; kc < ph.nkc; ++kc) {
-        uint32_t slot;
-        if (!acquire(slot)) return;
         const int kw = min(kChunk, ph.K - kc * kChunk);
-        const uint32_t bar = smem_u32(&c.full[slot]);
-        const uint32_t dst = smem_u32(c.ring + (size_t)slot * kStageBytes);
-        mbar_expect_tx(bar, 4u * (uint32_t)kw * 2u);
-#pragma unroll
-        for (int j = 0; j < 4; ++j)
-          bulk_g2s(dst + j * (kChunk * 2), rows[j] + (size_t)kc * kChunk, (uint32_t)kw * 2u, bar);
-        ++s;
+        for (int ww = 0; ww < nw; ++ww) {
+          uint32_t slot;
+          if (!acquire(slot)) return;
+          const uint32_t bar = smem_u32(&c.full[slot]);
+          if (lane == ww * 4) mbar_expect_tx(bar, 4u * (uint32_t)kw * 2u);
+          __syncwarp();
+          if (w == ww)
+            bulk_g2s(smem_u32(c.ring + (size_t)slot * kStageBytes) + j * (kChunk * 2),
+                     row + (size_t)kc * kChunk, (uint32_t)kw * 2u, bar);
+          ++s;
+        }
       }
     }
   }
   __device__ void att_phase(const AttSplit &a, int layer) {
     const FusedParams &p = *c.p;
     const Dims &dm = p.dm;
+    const int lane = threadIdx.x & 31;
     const int G = dm.Hq / dm.Hkv, qgroups = G / a.gq;
     for (int u = a.u0; u < a.u1 && ok; ++u) {
       const int stream = u / a.nch, chunk = u % a.nch;
@@ -264,16 +265,17 @@ struct Producer {
                           (size_t)chunk * a.CH) * dm.dh;
       const uint32_t bar = smem_u32(&c.full[slot]);
       const uint32_t dst = smem_u32(c.ring + (size_t)slot * kStageBytes);
-      mbar_expect_tx(bar, (uint32_t)kStageBytes);
-      bulk_g2s(dst, p.Kc + off, kStageBytes / 2, bar);
-      bulk_g2s(dst + kStageBytes / 2, p.Vc + off, kStageBytes / 2, bar);
+      if (lane == 0) mbar_expect_tx(bar, (uint32_t)kStageBytes);
+      __syncwarp();
+      if (lane == 0) bulk_g2s(dst, p.Kc + off, kStageBytes / 2, bar);
+      if (lane == 1) bulk_g2s(dst + kStageBytes / 2, p.Vc + off, kStageBytes / 2, bar);
       ++s;
     }
   }
 };
 
 // ---- consumer helpers ----------------------------------------------------------
-__device__ __forceinline__ float block_sum(const Ctx &c, float v) {
+__device__ __forceinline__ float block_sum(float v) {
   __shared__ float s_part[8];
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
@@ -286,105 +288,119 @@ __device__ __forceinline__ float block_sum(const Ctx &c, float v) {
   return t;
 }
 
-// position of element k of an activation vector in the permuted shared layout
+// position of element k of an activation vector in the permuted shared layout:
+// within each block of 256 elements, element lane*8 + j sits at (j/4)*128 + lane*4 + j%4
 __device__ __forceinline__ int act_index(int k) {
-  int kc = k / kChunk, e = k % kChunk;
-  return kc * kChunk + ((e & 7) >> 2) * 1024 + (e >> 3) * 4 + (e & 3);
+  return (k & ~255) + ((k & 7) >> 2) * 128 + ((k & 255) >> 3) * 4 + (k & 3);
 }
 
-// act := src (global fp32, length K), optionally RMS-normalised with `gain`
+// act := src (global fp32, length K).  With `gain` the vector (K <= 16 * 1024,
+// the model width) is RMS-normalised: one pass over L2, the values wait in
+// registers for the scale.
 __device__ void load_act(const Ctx &c, const float *src, int K, const bf16 *gain) {
   const int tid = threadIdx.x;
-  float scale = 1.f;
-  if (gain) {
-    float ss = 0.f;
-    for (int k = tid * 4; k < K; k += kConsumers * 4) {
-      float4 v = ldcg4(src + k);
-      ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
-    }
-    scale = rsqrtf(block_sum(c, ss) / (float)K + c.p->eps);
+  if (!gain) {
+#pragma unroll 4
+    for (int k = tid * 4; k < K; k += kConsumers * 4)
+      *reinterpret_cast<float4 *>(c.act + act_index(k)) = ldcg4(src + k);
+    consumer_sync();
+    return;
   }
-  for (int k = tid * 4; k < K; k += kConsumers * 4) {
-    float4 v = ldcg4(src + k);
-    if (gain) {
-      uint2 gw = *reinterpret_cast<const uint2 *>(gain + k);
-      v.x *= scale * bfl(gw.x); v.y *= scale * bfh(gw.x);
-      v.z *= scale * bfl(gw.y); v.w *= scale * bfh(gw.y);
+  constexpr int kMaxIt = 16;   // 16 * 1024 floats
+  float4 v[kMaxIt];
+  float ss = 0.f;
+#pragma unroll
+  for (int it = 0; it < kMaxIt; ++it) {
+    const int k = it * (kConsumers * 4) + tid * 4;
+    if (k < K) {
+      v[it] = ldcg4(src + k);
+      ss += v[it].x * v[it].x + v[it].y * v[it].y + v[it].z * v[it].z + v[it].w * v[it].w;
     }
-    *reinterpret_cast<float4 *>(c.act + act_index(k)) = v;
+  }
+  const float scale = rsqrtf(block_sum(ss) / (float)K + c.p->eps);
+#pragma unroll
+  for (int it = 0; it < kMaxIt; ++it) {
+    const int k = it * (kConsumers * 4) + tid * 4;
+    if (k < K) {
+      float4 t = v[it];
+      const uint2 gw = *reinterpret_cast<const uint2 *>(gain + k);
+      t.x *= scale * bfl(gw.x); t.y *= scale * bfh(gw.x);
+      t.z *= scale * bfl(gw.y); t.w *= scale * bfh(gw.y);
+      *reinterpret_cast<float4 *>(c.act + act_index(k)) = t;
+    }
   }
   consumer_sync();
 }
 
 struct Consumer {
   const Ctx &c;
-  uint32_t s;     // stages consumed so far
-  uint32_t rbuf;  // parity of the reduction buffer
-  bool ok;
-  __device__ Consumer(const Ctx &cc) : c(cc), s(0), rbuf(0), ok(true) {}
+  uint32_t s;     // ring stages of all finished phases (the same in every warp)
+  __device__ Consumer(const Ctx &cc) : c(cc), s(0) {}
 
-  __device__ __forceinline__ bool wait_stage(uint32_t &slot) {
+  // Wait until stage number `sn` (counted over the whole step) has landed.
+  // Stages of one slot are consumed by different warps, and a parity wait cannot
+  // tell fill k from fill k-2: so first wait until fill k-1 of the slot has been
+  // consumed (the producer issues fill k only after that), then for the parity.
+  // In abort mode both waits return at once and the (meaningless) work goes on.
+  __device__ __forceinline__ uint32_t wait_stage(uint32_t sn) {
     const uint32_t ns = (uint32_t)c.p->n_stages;
-    slot = s % ns;
-    // in abort mode the wait returns at once and the (meaningless) work goes on, so
-    // that every thread still reaches every barrier and the kernel ends
-    if (!wait_bar(c, smem_u32(&c.full[slot]), (s / ns) & 1u)) ok = false;
-    return true;
+    const uint32_t slot = sn % ns, fill = sn / ns;
+    if (c.released[slot] < fill && !*c.abort_flag) {
+      const uint64_t t0 = now_ns();
+      for (uint32_t it = 1; c.released[slot] < fill && !*c.abort_flag; ++it)
+        if ((it & 63u) == 0u && now_ns() - t0 > c.p->wait_ns) raise_timeout(c);
+    }
+    wait_bar(c, smem_u32(&c.full[slot]), fill & 1u);
+    return slot;
   }
-  __device__ __forceinline__ void release_stage(uint32_t slot) {
+  // the warp that consumed stage `sn` hands the slot back to the producer
+  __device__ __forceinline__ void release_stage(uint32_t slot, uint32_t sn) {
     __syncwarp();
-    if ((threadIdx.x & 31) == 0) mbar_arrive(smem_u32(&c.empty[slot]));
-    ++s;
+    if ((threadIdx.x & 31) == 0) {
+      c.released[slot] = sn / (uint32_t)c.p->n_stages + 1u;
+      mbar_arrive(smem_u32(&c.empty[slot]));
+    }
   }
 
   // One GEMV phase over the activation vector held in c.act.
   __device__ void gemv_phase(const Phase &ph, int layer) {
-    const FusedParams &p = *c.p;
-    const Dims &dm = p.dm;
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    for (int g = ph.g0; g < ph.g1; ++g) {
-      float acc[4] = {0.f, 0.f, 0.f, 0.f};
-      for (int kc = 0; kc < ph.nkc; ++kc) {
-        uint32_t slot;
-        wait_stage(slot);
-        const int kw = min(kChunk, ph.K - kc * kChunk);
-        if (tid * 8 < kw) {
-          const unsigned char *st = c.ring + (size_t)slot * kStageBytes + tid * 16;
-          const float *a = c.act + kc * kChunk + tid * 4;
-          const float4 x0 = *reinterpret_cast<const float4 *>(a);
-          const float4 x1 = *reinterpret_cast<const float4 *>(a + 1024);
+    const Dims &dm = c.p->dm;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    for (int S0 = ph.g0; S0 < ph.g1; S0 += 8) {
+      const int nw = min(8, ph.g1 - S0);
+      if (warp < nw) {
+        float acc[4] = {0.f, 0.f, 0.f, 0.f};
+        const uint32_t first = s + (uint32_t)(S0 - ph.g0) * (uint32_t)ph.nkc + (uint32_t)warp;
+        for (int kc = 0; kc < ph.nkc; ++kc) {
+          const uint32_t sn = first + (uint32_t)(kc * nw);
+          const uint32_t slot = wait_stage(sn);
+          const int kw = min(kChunk, ph.K - kc * kChunk);
+          const unsigned char *st = c.ring + (size_t)slot * kStageBytes + lane * 16;
+          const float *a = c.act + kc * kChunk + lane * 4;
+#pragma unroll 2
+          for (int b = 0; b < kChunk / 256; ++b) {
+            if (b * 256 + lane * 8 < kw) {
+              const float4 x0 = *reinterpret_cast<const float4 *>(a + b * 256);
+              const float4 x1 = *reinterpret_cast<const float4 *>(a + b * 256 + 128);
 #pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            const uint4 w = *reinterpret_cast<const uint4 *>(st + j * (kChunk * 2));
-            acc[j] += bfl(w.x) * x0.x + bfh(w.x) * x0.y + bfl(w.y) * x0.z + bfh(w.y) * x0.w +
-                      bfl(w.z) * x1.x + bfh(w.z) * x1.y + bfl(w.w) * x1.z + bfh(w.w) * x1.w;
+              for (int j = 0; j < 4; ++j) {
+                const uint4 w = *reinterpret_cast<const uint4 *>(st + j * (kChunk * 2) + b * 512);
+                acc[j] += bfl(w.x) * x0.x + bfh(w.x) * x0.y + bfl(w.y) * x0.z + bfh(w.y) * x0.w +
+                          bfl(w.z) * x1.x + bfh(w.z) * x1.y + bfl(w.w) * x1.z + bfh(w.w) * x1.w;
+              }
+            }
           }
+          release_stage(slot, sn);
         }
-        release_stage(slot);
-      }
-      // block reduction of the four sums, then the epilogue of the group
 #pragma unroll
-      for (int j = 0; j < 4; ++j) {
+        for (int j = 0; j < 4; ++j) {
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) acc[j] += __shfl_xor_sync(0xffffffffu, acc[j], o);
-      }
-      if (lane == 0) {
-#pragma unroll
-        for (int j = 0; j < 4; ++j) c.red[rbuf][warp][j] = acc[j];
-      }
-      consumer_sync();
-      if (warp == 0) {
-        float y = 0.f;
-        if (lane < 4) {
-#pragma unroll
-          for (int w = 0; w < 8; ++w) y += c.red[rbuf][w][lane];
+          for (int o = 16; o > 0; o >>= 1) acc[j] += __shfl_xor_sync(0xffffffffu, acc[j], o);
         }
-        const float y0 = __shfl_sync(0xffffffffu, y, 0), y1 = __shfl_sync(0xffffffffu, y, 1);
-        const float y2 = __shfl_sync(0xffffffffu, y, 2), y3 = __shfl_sync(0xffffffffu, y, 3);
-        if (lane == 0) epilogue(ph, dm, layer, g, y0, y1, y2, y3);
+        if (lane == 0) epilogue(ph, dm, layer, S0 + warp, acc[0], acc[1], acc[2], acc[3]);
       }
-      rbuf ^= 1u;
     }
+    s += (uint32_t)(ph.g1 - ph.g0) * (uint32_t)ph.nkc;
   }
 
   __device__ void epilogue(const Phase &ph, const Dims &dm, int layer, int g, float y0, float y1, float y2,
@@ -430,19 +446,24 @@ struct Consumer {
     }
   }
 
-  // Attention of this CTA's units; writes one partial (max, sum, o) per stream
-  // segment: part[(stream * ncta + cta)][gq][dh + 2].
+  // Attention of this CTA's units.  Each stream segment yields one partial
+  // (max, sum, o) in part[(stream * ncta + cta)][gq][dh + 2]; the CTA whose
+  // arrival completes a stream merges the stream's partials into attn_out.
   template <int DH, int GQ>
-  __device__ void att_phase(const AttSplit &a, int layer) {
+  __device__ void att_phase(const AttSplit &a, int layer, unsigned ordinal) {
     const FusedParams &p = *c.p;
     const Dims &dm = p.dm;
     constexpr int EPL = DH / 8;
+    __shared__ int s_nseg, s_last;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, part = lane & 7;
     const int worker = warp * 4 + (lane >> 3);
+    // the 8 lanes of a worker run the position loop in lockstep; other workers of
+    // the warp may run fewer iterations, so in-loop shuffles name only the worker
     const unsigned wmask = 0xffu << (lane & 24);
     const int G = dm.Hq / dm.Hkv, qgroups = G / GQ;
     const float scale = rsqrtf((float)DH);
     int u = a.u0;
+    uint32_t ring_k = 0;   // ring stages of this phase seen so far (every warp counts them all)
     while (u < a.u1) {
       const int stream = u / a.nch;
       const int kvh = stream / qgroups, qg = stream % qgroups;
@@ -461,20 +482,29 @@ struct Consumer {
       for (; u < u_end; ++u) {
         const int chunk = u % a.nch;
         const bool tail = chunk == a.nch - 1;
-        uint32_t slot = 0;
-        if (!tail) wait_stage(slot);
+        // a ring stage belongs to one warp (its 4 workers walk the CH positions); the
+        // tail chunk is read from global memory by all 32 workers
+        uint32_t slot = 0, sn = 0;
+        bool mine = true;
+        if (!tail) {
+          mine = (ring_k & 7u) == (uint32_t)warp;
+          sn = s + ring_k;
+          if (mine) slot = wait_stage(sn);
+          ++ring_k;
+        }
         const int t0 = chunk * a.CH;
-        const int cnt = tail ? (p.pos - t0 + 1) : a.CH;
+        const int cnt = tail ? (p.pos - t0 + 1) : (mine ? a.CH : 0);
+        const int i0 = tail ? worker : (lane >> 3), istep = tail ? 32 : 4;
         const size_t goff = ((((size_t)layer * dm.max_slots + p.slot) * dm.Hkv + kvh) * dm.max_seq + t0) * DH;
-        for (int i = worker; i < cnt; i += 32) {
+        for (int i = i0; i < cnt; i += istep) {
           float kf[EPL], vf[EPL];
           if (tail) {
             const bf16 *kp = p.Kc + goff + (size_t)i * DH + part * EPL;
             const bf16 *vp = p.Vc + goff + (size_t)i * DH + part * EPL;
 #pragma unroll
             for (int e = 0; e < EPL; e += 4) {
-              uint2 kw = __ldcg(reinterpret_cast<const uint2 *>(kp + e));
-              uint2 vw = __ldcg(reinterpret_cast<const uint2 *>(vp + e));
+              const uint2 kw = __ldcg(reinterpret_cast<const uint2 *>(kp + e));
+              const uint2 vw = __ldcg(reinterpret_cast<const uint2 *>(vp + e));
               kf[e] = bfl(kw.x); kf[e + 1] = bfh(kw.x); kf[e + 2] = bfl(kw.y); kf[e + 3] = bfh(kw.y);
               vf[e] = bfl(vw.x); vf[e + 1] = bfh(vw.x); vf[e + 2] = bfl(vw.y); vf[e + 3] = bfh(vw.y);
             }
@@ -483,8 +513,8 @@ struct Consumer {
             const unsigned char *vs = ks + kStageBytes / 2;
 #pragma unroll
             for (int e = 0; e < EPL; e += 4) {
-              uint2 kw = *reinterpret_cast<const uint2 *>(ks + e * 2);
-              uint2 vw = *reinterpret_cast<const uint2 *>(vs + e * 2);
+              const uint2 kw = *reinterpret_cast<const uint2 *>(ks + e * 2);
+              const uint2 vw = *reinterpret_cast<const uint2 *>(vs + e * 2);
               kf[e] = bfl(kw.x); kf[e + 1] = bfh(kw.x); kf[e + 2] = bfl(kw.y); kf[e + 3] = bfh(kw.y);
               vf[e] = bfl(vw.x); vf[e + 1] = bfh(vw.x); vf[e + 2] = bfl(vw.y); vf[e + 3] = bfh(vw.y);
             }
@@ -505,7 +535,7 @@ struct Consumer {
             for (int e = 0; e < EPL; ++e) o[g][e] = o[g][e] * corr + pr * vf[e];
           }
         }
-        if (!tail) release_stage(slot);
+        if (!tail && mine) release_stage(slot, sn);
       }
       // merge the 32 workers: 4 per warp by shuffles, 8 warps through shared memory
 #pragma unroll
@@ -526,9 +556,13 @@ struct Consumer {
           mx[g] = mn;
         }
       }
+      // the activation buffer is free during attention: it holds the merge scratch
       float *s_o = c.act;                       // [8][GQ][DH]
       float *s_ml = c.act + 8 * GQ * DH;        // [8][GQ][2]
-      consumer_sync();                          // the activation buffer is free during attention
+      int *s_list = reinterpret_cast<int *>(c.act + 8 * GQ * (DH + 2));   // CTAs holding a partial
+      float *s_pm = c.act + 8 * GQ * (DH + 2) + kFusedMaxCtas;            // [seg][kMaxGQ] max
+      float *s_pl = s_pm + kFusedMaxCtas * kMaxGQ;                        // [seg][kMaxGQ] sum
+      consumer_sync();
       if (lane < 8) {
 #pragma unroll
         for (int g = 0; g < GQ; ++g) {
@@ -556,38 +590,47 @@ struct Consumer {
         if (e == 0) { dst[g * (DH + 2) + DH] = M; dst[g * (DH + 2) + DH + 1] = Ls; }
       }
       consumer_sync();
-    }
-  }
-
-  // act := attention output of all heads, merged from the partials of all CTAs
-  template <int DH, int GQ>
-  __device__ void combine_to_act(const AttSplit &a) {
-    const FusedParams &p = *c.p;
-    const Dims &dm = p.dm;
-    const int G = dm.Hq / dm.Hkv, qgroups = G / GQ;
-    for (int i = threadIdx.x; i < dm.Hq * DH; i += kConsumers) {
-      const int h = i / DH, e = i % DH;
-      const int kvh = h / G, qg = (h % G) / GQ, g = (h % G) % GQ;
-      const int stream = kvh * qgroups + qg;
-      const int c0 = cta_of_unit(stream * a.nch, a.units, c.ncta);
-      const int c1 = cta_of_unit((stream + 1) * a.nch - 1, a.units, c.ncta);
-      // CTAs c0..c1 hold the stream's units; one with an empty range wrote nothing
-      float M = -INFINITY;
-      for (int cc = c0; cc <= c1; ++cc) {
-        if ((long long)a.units * cc / c.ncta == (long long)a.units * (cc + 1) / c.ncta) continue;
-        M = fmaxf(M, __ldcg(p.part + ((size_t)stream * c.ncta + cc) * (GQ * (DH + 2)) + g * (DH + 2) + DH));
+      // Publish the partial.  The CTA whose arrival completes the stream merges all
+      // of the stream's partials into attn_out; the others go on to the barrier.
+      if (tid == 0) {
+        const int c0 = cta_of_unit(stream * a.nch, a.units, c.ncta);
+        const int c1 = cta_of_unit((stream + 1) * a.nch - 1, a.units, c.ncta);
+        int nseg = 0;
+        for (int cc = c0; cc <= c1; ++cc)   // a CTA with an empty range wrote nothing
+          if ((long long)a.units * cc / c.ncta != (long long)a.units * (cc + 1) / c.ncta) s_list[nseg++] = cc;
+        __threadfence();
+        const unsigned old = atomicAdd(p.stream_count + stream, 1u);
+        s_nseg = nseg;
+        s_last = (old + 1u == (unsigned)nseg * ordinal) ? 1 : 0;
       }
-      float Ls = 0.f, O = 0.f;
-      for (int cc = c0; cc <= c1; ++cc) {
-        if ((long long)a.units * cc / c.ncta == (long long)a.units * (cc + 1) / c.ncta) continue;
-        const float *src = p.part + ((size_t)stream * c.ncta + cc) * (GQ * (DH + 2)) + g * (DH + 2);
-        const float cf = __expf(__ldcg(src + DH) - M);
-        Ls += __ldcg(src + DH + 1) * cf;
-        O += __ldcg(src + e) * cf;
+      consumer_sync();
+      if (s_last) {
+        __threadfence();
+        const int nseg = s_nseg;
+        for (int i = tid; i < nseg * GQ; i += kConsumers) {
+          const int sg = i / GQ, g = i % GQ;
+          const float *src = p.part + ((size_t)stream * c.ncta + s_list[sg]) * (GQ * (DH + 2)) + g * (DH + 2);
+          s_pm[sg * kMaxGQ + g] = __ldcg(src + DH);
+          s_pl[sg * kMaxGQ + g] = __ldcg(src + DH + 1);
+        }
+        consumer_sync();
+        for (int i = tid; i < GQ * DH; i += kConsumers) {
+          const int g = i / DH, e = i % DH;
+          float M = -INFINITY;
+          for (int sg = 0; sg < nseg; ++sg) M = fmaxf(M, s_pm[sg * kMaxGQ + g]);
+          float Ls = 0.f, O = 0.f;
+#pragma unroll 4
+          for (int sg = 0; sg < nseg; ++sg) {
+            const float cf = __expf(s_pm[sg * kMaxGQ + g] - M);
+            Ls += s_pl[sg * kMaxGQ + g] * cf;
+            O += __ldcg(p.part + ((size_t)stream * c.ncta + s_list[sg]) * (GQ * (DH + 2)) + g * (DH + 2) + e) * cf;
+          }
+          p.attn_out[(h0 + g) * DH + e] = O / Ls;
+        }
       }
-      c.act[act_index(i)] = O / Ls;
+      consumer_sync();
     }
-    consumer_sync();
+    s += ring_k;
   }
 };
 
@@ -595,7 +638,7 @@ template <int DH, int GQ>
 __global__ void __launch_bounds__(kFusedThreads, 1) k_step_b1(const __grid_constant__ FusedParams p) {
   extern __shared__ __align__(128) unsigned char smem[];
   __shared__ __align__(8) uint64_t s_full[kMaxStages], s_empty[kMaxStages];
-  __shared__ float s_red[2][8][4];
+  __shared__ uint32_t s_released[kMaxStages];
   __shared__ int s_abort;
   const int tid = threadIdx.x, warp = tid >> 5;
   Ctx c;
@@ -603,14 +646,15 @@ __global__ void __launch_bounds__(kFusedThreads, 1) k_step_b1(const __grid_const
   c.ring = smem;
   c.act = reinterpret_cast<float *>(smem + (size_t)p.n_stages * kStageBytes);
   c.full = s_full; c.empty = s_empty;
+  c.released = s_released;
   c.abort_flag = &s_abort;
-  c.red = s_red;
   c.cta = blockIdx.x; c.ncta = gridDim.x;
   if (tid == 0) {
     s_abort = 0;
     for (int i = 0; i < p.n_stages; ++i) {
+      s_released[i] = 0;
       mbar_init(smem_u32(&s_full[i]), 1);
-      mbar_init(smem_u32(&s_empty[i]), 8);
+      mbar_init(smem_u32(&s_empty[i]), 1);   // released by the one warp that consumed the stage
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -630,26 +674,24 @@ __global__ void __launch_bounds__(kFusedThreads, 1) k_step_b1(const __grid_const
 
   if (warp == 8) {
     // ------------------------------------------------------------ producer
-    if ((tid & 31) == 0) {
-      Producer pr(c);
-      for (int l = 0; l < L && pr.ok; ++l) {
-        if (lo <= l && l < hi) continue;
-        pr.gemv_phase(make_phase(p, PH_QKV, l, c.cta, c.ncta));
-        pr.att_phase(att, l);
-        pr.gemv_phase(make_phase(p, PH_OPROJ, l, c.cta, c.ncta));
-        pr.gemv_phase(make_phase(p, PH_GATEUP, l, c.cta, c.ncta));
-        pr.gemv_phase(make_phase(p, PH_DOWN, l, c.cta, c.ncta));
-      }
-      if (pr.ok && p.logits) pr.gemv_phase(make_phase(p, PH_HEAD, 0, c.cta, c.ncta));
-      if (!pr.ok) {
-        // drain: wait (bounded) until every copy already issued has landed
-        const uint32_t ns = (uint32_t)p.n_stages;
-        const uint32_t first = pr.s > ns ? pr.s - ns : 0;
-        for (uint32_t s = first; s < pr.s; ++s) {
-          const uint32_t bar = smem_u32(&s_full[s % ns]);
-          const uint64_t t0 = now_ns();
-          while (!mbar_try_wait(bar, (s / ns) & 1u) && now_ns() - t0 < p.wait_ns) {}
-        }
+    Producer pr(c);
+    for (int l = 0; l < L && pr.ok; ++l) {
+      if (lo <= l && l < hi) continue;
+      pr.gemv_phase(make_phase(p, PH_QKV, l, c.cta, c.ncta));
+      pr.att_phase(att, l);
+      pr.gemv_phase(make_phase(p, PH_OPROJ, l, c.cta, c.ncta));
+      pr.gemv_phase(make_phase(p, PH_GATEUP, l, c.cta, c.ncta));
+      pr.gemv_phase(make_phase(p, PH_DOWN, l, c.cta, c.ncta));
+    }
+    if (pr.ok && p.logits) pr.gemv_phase(make_phase(p, PH_HEAD, 0, c.cta, c.ncta));
+    if (!pr.ok && (tid & 31) == 0) {
+      // drain: wait (bounded) until every copy already issued has landed
+      const uint32_t ns = (uint32_t)p.n_stages;
+      const uint32_t first = pr.s > ns ? pr.s - ns : 0;
+      for (uint32_t s = first; s < pr.s; ++s) {
+        const uint32_t bar = smem_u32(&s_full[s % ns]);
+        const uint64_t t0 = now_ns();
+        while (!mbar_try_wait(bar, (s / ns) & 1u) && now_ns() - t0 < p.wait_ns) {}
       }
     }
     return;
@@ -664,50 +706,75 @@ __global__ void __launch_bounds__(kFusedThreads, 1) k_step_b1(const __grid_const
     for (int l = 0; l < L; ++l) s->m[l] = (lo <= l && l < hi) ? 0 : 1;
     s->rows_layers = n; s->layers_touched = n;
   }
-  // embedding row -> residual stream (CTA 0 publishes it; everybody normalises its own copy)
+  // embedding row -> residual stream (CTA 0 publishes it)
   const Dims &dm = p.dm;
   if (c.cta == 0) {
     const bf16 *e = p.embed + (size_t)tok * dm.d;
     for (int k = tid * 8; k < dm.d; k += kConsumers * 8) {
-      uint4 w = *reinterpret_cast<const uint4 *>(e + k);
+      const uint4 w = *reinterpret_cast<const uint4 *>(e + k);
       *reinterpret_cast<float4 *>(p.x + k) = make_float4(bfl(w.x), bfh(w.x), bfl(w.y), bfh(w.y));
       *reinterpret_cast<float4 *>(p.x + k + 4) = make_float4(bfl(w.z), bfh(w.z), bfl(w.w), bfh(w.w));
     }
   }
   Consumer cs(c);
-  unsigned bidx = 0;
+  unsigned bidx = 0, ordinal = 0;
+  // optional phase timer (thread 0 of every CTA): cycles spent up to each phase boundary
+  const bool timing = p.phase_cycles != nullptr && tid == 0;
+  long long t_prev = clock64();
+  auto tick = [&](int k) {
+    if (timing) {
+      const long long t = clock64();
+      p.phase_cycles[c.cta * kFusedPhases + k] += t - t_prev;
+      t_prev = t;
+    }
+  };
   grid_barrier(c, ++bidx);
+  tick(0);
   for (int l = 0; l < L; ++l) {
     if (lo <= l && l < hi) continue;   // dropped block: the hidden state passes through
     load_act(c, p.x, dm.d, p.layers[l].attn_norm);
+    tick(1);
     cs.gemv_phase(make_phase(p, PH_QKV, l, c.cta, c.ncta), l);
+    tick(2);
     grid_barrier(c, ++bidx);
-    cs.template att_phase<DH, GQ>(att, l);
+    tick(3);
+    cs.template att_phase<DH, GQ>(att, l, ++ordinal);
+    tick(4);
     grid_barrier(c, ++bidx);
-    cs.template combine_to_act<DH, GQ>(att);
+    tick(3);
+    load_act(c, p.attn_out, dm.Hq * dm.dh, nullptr);
+    tick(1);
     cs.gemv_phase(make_phase(p, PH_OPROJ, l, c.cta, c.ncta), l);
+    tick(5);
     grid_barrier(c, ++bidx);
+    tick(3);
     load_act(c, p.x, dm.d, p.layers[l].mlp_norm);
+    tick(1);
     cs.gemv_phase(make_phase(p, PH_GATEUP, l, c.cta, c.ncta), l);
+    tick(6);
     grid_barrier(c, ++bidx);
+    tick(3);
     load_act(c, p.u, dm.f, nullptr);
+    tick(1);
     cs.gemv_phase(make_phase(p, PH_DOWN, l, c.cta, c.ncta), l);
+    tick(7);
     grid_barrier(c, ++bidx);
+    tick(3);
   }
   // KV fill by copy for the dropped blocks: CTA j takes block lo + j, lo + j + ncta, ...
   if (p.kv_fill == D3_FILL_COPY) {
     const int nkv = dm.Hkv * dm.dh;
+    unsigned short *Ku = reinterpret_cast<unsigned short *>(p.Kc);
+    unsigned short *Vu = reinterpret_cast<unsigned short *>(p.Vc);
     for (int l = lo + c.cta; l < hi; l += c.ncta) {
       for (int i = tid; i < nkv; i += kConsumers) {
         const int h = i / dm.dh, e = i % dm.dh;
         const size_t dst = ((((size_t)l * dm.max_slots + p.slot) * dm.Hkv + h) * dm.max_seq + p.pos) * dm.dh + e;
         if (lo == 0) {
-          p.Kc[dst] = __float2bfloat16_rn(0.f);
-          p.Vc[dst] = __float2bfloat16_rn(0.f);
+          Ku[dst] = 0;
+          Vu[dst] = 0;
         } else {
           const size_t src = ((((size_t)(lo - 1) * dm.max_slots + p.slot) * dm.Hkv + h) * dm.max_seq + p.pos) * dm.dh + e;
-          unsigned short *Ku = reinterpret_cast<unsigned short *>(p.Kc);
-          unsigned short *Vu = reinterpret_cast<unsigned short *>(p.Vc);
           Ku[dst] = __ldcg(Ku + src);   // written by another CTA earlier in this kernel
           Vu[dst] = __ldcg(Vu + src);
         }
@@ -718,13 +785,13 @@ __global__ void __launch_bounds__(kFusedThreads, 1) k_step_b1(const __grid_const
     load_act(c, p.x, dm.d, p.final_norm);
     cs.gemv_phase(make_phase(p, PH_HEAD, 0, c.cta, c.ncta), 0);
   }
+  tick(8);
 }
 
 }  // namespace
 
 // ------------------------------------------------------------------ host side
 struct FusedPlan {
-  int ok;            // 1 when the fused kernel serves this model
   int grid, n_stages, act_floats;
   size_t smem;
   void *func;
@@ -732,18 +799,17 @@ struct FusedPlan {
 
 template <int DH, int GQ>
 static bool try_plan(FusedPlan &pl, const d3_config &c) {
-  int dev = 0, sms = 0, optin = 0;
+  int dev = 0, sms = 0, optin = 0, coop = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return false;
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
-  int coop = 0;
   cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev);
   if (!coop || sms < 1) return false;
   int need = c.d_model;
   if (c.d_ffn > need) need = c.d_ffn;
   if (c.n_q_heads * c.head_dim > need) need = c.n_q_heads * c.head_dim;
   need = (need + kChunk - 1) / kChunk * kChunk;
-  const int att_need = 8 * kMaxGQ * (128 + 2);
+  const int att_need = 8 * kMaxGQ * (128 + 2) + kFusedMaxCtas * (1 + 2 * kMaxGQ);
   if (need < att_need) need = (att_need + kChunk - 1) / kChunk * kChunk;
   const int reserve = 4096;   // static shared memory of the kernel and slack
   int stages = (optin - reserve - need * 4) / kStageBytes;
@@ -761,8 +827,7 @@ static bool try_plan(FusedPlan &pl, const d3_config &c) {
           cudaSuccess ||
       per_sm < 1)
     return false;
-  pl.grid = sms;
-  pl.ok = 1;
+  pl.grid = sms < kFusedMaxCtas ? sms : kFusedMaxCtas;
   return true;
 }
 
@@ -772,7 +837,7 @@ int fused_plan(const d3_config &c, int *grid, int *n_stages, int *act_floats, si
   const int G = c.n_q_heads / c.n_kv_heads;
   const int gq = (G % 4 == 0) ? 4 : (G % 2 == 0) ? 2 : 1;
   bool ok = false;
-  if (c.vocab % 4 == 0 && c.head_dim * 2 * c.max_seq % 16 == 0) {
+  if (c.vocab % 4 == 0 && c.d_model <= 16 * 1024) {
     if (c.head_dim == 128 && gq == 1) ok = try_plan<128, 1>(pl, c);
     else if (c.head_dim == 128 && gq == 4) ok = try_plan<128, 4>(pl, c);
     else if (c.head_dim == 64 && gq == 1) ok = try_plan<64, 1>(pl, c);
@@ -785,7 +850,8 @@ int fused_plan(const d3_config &c, int *grid, int *n_stages, int *act_floats, si
 }
 
 int launch_fused_step(void *func, int grid, size_t smem, FusedParams &fp, cudaStream_t st) {
-  if (cudaMemsetAsync(fp.bar_counter, 0, sizeof(unsigned), st) != cudaSuccess) return -1;
+  // grid-barrier counter and per-stream arrival counters start every step at zero
+  if (cudaMemsetAsync(fp.bar_counter, 0, kFusedSyncBytes, st) != cudaSuccess) return -1;
   void *args[] = {(void *)&fp};
   if (cudaLaunchCooperativeKernel(func, dim3(grid), dim3(kFusedThreads), args, smem, st) != cudaSuccess)
     return -1;

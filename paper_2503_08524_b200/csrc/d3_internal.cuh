@@ -78,6 +78,8 @@ struct LayerPtrs {
 };
 
 static constexpr int kFusedMaxCtas = 192;
+static constexpr int kFusedSyncBytes = 1024;   // grid-barrier counter + per-stream arrival counters
+static constexpr int kFusedPhases = 9;         // timed phases of the fused kernel
 
 // parameters of the fused batch-1 step kernel (passed by value)
 struct FusedParams {
@@ -92,8 +94,10 @@ struct FusedParams {
   bf16 *Kc, *Vc;
   const float2 *rope;
   DevSched *sched;
-  unsigned *bar_counter;
-  float *x, *qkv, *u, *part;
+  unsigned *bar_counter;        // grid barrier
+  unsigned *stream_count;       // arrivals per attention stream
+  long long *phase_cycles;      // nullable: [cta][kFusedPhases] cycles per phase
+  float *x, *qkv, *u, *part, *attn_out;
   float *logits;
   int32_t n_stages, act_floats;
   unsigned long long wait_ns;   // bound of every device-side wait
@@ -101,7 +105,7 @@ struct FusedParams {
 
 // Byte offsets of the regions of the caller's scratch buffer.
 struct Layout {
-  size_t sched, rope, x, qkv, attn_out, part_o, part_ml, u, layer_tab, bar, part_fused, total;
+  size_t sched, rope, x, qkv, attn_out, part_o, part_ml, u, layer_tab, bar, phase, part_fused, total;
   int max_splits;
 };
 

@@ -88,6 +88,7 @@ def test_tiny_generate_teacher_forced(B, shape, alpha, kv_round, exec_mode):
         assert st["n"][0] == O.window(shape.n_layers, alpha, i, 0)[0]
         layers += st["rows_layers"]
         tok = O.argmax(r["logits"][0])
+    gpu.d3_sync()
     assert layers == sum(O.depth(shape.n_layers, alpha, i) for i in range(1, 32))
     assert gpu.d3_slot_pos(1) == orc.slot_pos(1) == 16 + 31
     gpu.close()
@@ -256,6 +257,7 @@ def test_production_widths(B, base, layers, Bn):
         r = orc.decode_step(list(range(Bn)), toks, gi, alpha)
         g = gpu.d3_decode_step(list(range(Bn)), toks, gi, alpha)
         check_step(f"step {step}", g.cpu().numpy(), gpu.d3_read_hidden(Bn), r["logits"], r["hidden"])
+    gpu.d3_sync()          # raises on a deferred device status (a bounded wait that ran out)
     gpu.close()
 
 
