@@ -178,7 +178,7 @@ int32_t d3_set_exec(d3_model *m, int32_t mode);
  * steps are slower end to end; totals accumulate until read.
  * d3_read_profile: ms[k], launches[k] for k < D3_PROF_KINDS (HOST arrays), then
  * clears the totals.  d3_profile_name(k): a static string. */
-#define D3_PROF_KINDS 21   /* 10 kernel classes + 11 figures from inside the single-kernel step */
+#define D3_PROF_KINDS 22   /* 10 kernel classes + 12 figures from inside the single-kernel step */
 #define D3_PROF_FUSED0 10
 int32_t d3_profile(d3_model *m, int32_t enable);
 int32_t d3_read_profile(d3_model *m, float *ms, int32_t *launches);

@@ -123,7 +123,7 @@ static const char *kProfNames[D3_PROF_KINDS] = {
     "down+resid", "kv_fill", "norm+lm_head", "fused_step",
     // phases inside the fused step kernel (mean over CTAs, nominal-clock ms)
     "fused:prologue", "fused:load_act", "fused:qkv", "fused:grid_barriers", "fused:attention",
-    "fused:o_proj", "fused:gate_up", "fused:down", "fused:head+fill",
+    "fused:o_proj", "fused:gate_up", "fused:down", "fused:head+fill", "fused:ring_wait(warp0)",
     // smallest and largest per-CTA time spent in grid barriers
     "fused:grid_barriers_min", "fused:grid_barriers_max"};
 

@@ -25,6 +25,8 @@
 // abort mode: waits return at once, the producer stops issuing and drains the
 // copies in flight, and every thread still walks the same control flow to the
 // end so that no barrier is left waiting.
+#include <stdlib.h>
+
 #include "d3_internal.cuh"
 
 namespace d3 {
@@ -335,7 +337,8 @@ __device__ void load_act(const Ctx &c, const float *src, int K, const bf16 *gain
 struct Consumer {
   const Ctx &c;
   uint32_t s;     // ring stages of all finished phases (the same in every warp)
-  __device__ Consumer(const Ctx &cc) : c(cc), s(0) {}
+  long long ring_wait;   // cycles this thread spent waiting for ring stages (timing runs)
+  __device__ Consumer(const Ctx &cc) : c(cc), s(0), ring_wait(0) {}
 
   // Wait until stage number `sn` (counted over the whole step) has landed.
   // Stages of one slot are consumed by different warps, and a parity wait cannot
@@ -345,12 +348,14 @@ struct Consumer {
   __device__ __forceinline__ uint32_t wait_stage(uint32_t sn) {
     const uint32_t ns = (uint32_t)c.p->n_stages;
     const uint32_t slot = sn % ns, fill = sn / ns;
+    const long long tw = clock64();
     if (c.released[slot] < fill && !*c.abort_flag) {
       const uint64_t t0 = now_ns();
       for (uint32_t it = 1; c.released[slot] < fill && !*c.abort_flag; ++it)
         if ((it & 63u) == 0u && now_ns() - t0 > c.p->wait_ns) raise_timeout(c);
     }
     wait_bar(c, smem_u32(&c.full[slot]), fill & 1u);
+    ring_wait += clock64() - tw;
     return slot;
   }
   // the warp that consumed stage `sn` hands the slot back to the producer
@@ -786,6 +791,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) k_step_b1(const __grid_const
     cs.gemv_phase(make_phase(p, PH_HEAD, 0, c.cta, c.ncta), 0);
   }
   tick(8);
+  if (timing) p.phase_cycles[c.cta * kFusedPhases + 9] += cs.ring_wait;
 }
 
 }  // namespace
@@ -814,6 +820,10 @@ static bool try_plan(FusedPlan &pl, const d3_config &c) {
   const int reserve = 4096;   // static shared memory of the kernel and slack
   int stages = (optin - reserve - need * 4) / kStageBytes;
   if (stages > kMaxStages) stages = kMaxStages;
+  if (const char *env = getenv("D3_FUSED_STAGES")) {   // tuning knob: a shallower ring
+    const int want = atoi(env);
+    if (want >= 3 && want < stages) stages = want;
+  }
   if (stages < 3) return false;
   pl.n_stages = stages;
   pl.act_floats = need;

@@ -79,7 +79,7 @@ struct LayerPtrs {
 
 static constexpr int kFusedMaxCtas = 192;
 static constexpr int kFusedSyncBytes = 1024;   // grid-barrier counter + per-stream arrival counters
-static constexpr int kFusedPhases = 9;         // timed phases of the fused kernel
+static constexpr int kFusedPhases = 10;        // timed phases of the fused kernel (+ ring wait)
 
 // parameters of the fused batch-1 step kernel (passed by value)
 struct FusedParams {
