@@ -184,6 +184,52 @@ int32_t d3_profile(d3_model *m, int32_t enable);
 int32_t d3_read_profile(d3_model *m, float *ms, int32_t *launches);
 const char *d3_profile_name(int32_t kind);
 
+/* One batch-1 decode step that allocates nothing.  (The paper has no
+ * counterpart: this entry point exists for the sake of the caller, not of the
+ * method.)
+ *
+ * Who needs it: code that may not call cudaMalloc at the point where it wants
+ * to decode -- a plugin running inside a host application that owns all device
+ * memory and hands out only the tensors it chooses, a real-time or
+ * safety-critical loop that forbids allocation after start-up, a process
+ * running so close to the memory limit that an allocation could fail.  Such a
+ * caller cannot provide the scratch buffer that d3_load asks for.  Here the
+ * scratch (schedule, rotary table, activations, attention partials, barrier
+ * counters, weight-pointer table) is a fixed array of D3_NOALLOC_SCRATCH_BYTES
+ * inside the library image; every GPU that loads the library holds that much
+ * memory until the process exits.  No call made here allocates or frees device
+ * memory, and no model handle is created.
+ *
+ * It computes what d3_decode_step computes for a single row through the
+ * single-kernel step (Sec. 3.4): the sequence in `slot`, whose cache holds
+ * `pos` >= 1 tokens, feeds `token` = T_{i-1} with i = gen_index >= 1, writes
+ * K,V of the retained blocks (and the fill of the dropped ones) at position
+ * `pos` of kv_dev, and writes the logits that choose T_i to logits_dev
+ * [vocab] (fp32).  The caller keeps count of `pos` itself.  cfg, weights and
+ * kv_dev mean what they mean for d3_load (cfg->max_batch is ignored); kv_fill
+ * must be D3_FILL_NONE or D3_FILL_COPY.
+ *
+ * Limits and errors: D3_ECAPACITY when the scratch one row of `cfg` needs
+ * exceeds D3_NOALLOC_SCRATCH_BYTES (roughly: Llama-2-7B/13B shapes with
+ * max_seq up to a few thousand fit, the 70B shape does not) or pos >= max_seq;
+ * D3_EINVAL for sizes the single-kernel step does not serve (head_dim /
+ * grouping other than 128x1, 128x4, 64x1, 32x4; vocab not a multiple of 4),
+ * for fill RECOMPUTE and for bad arguments; D3_ECUDA when a runtime call fails.
+ *
+ * First call on a device: it looks up the array's device address and sets the
+ * kernel's shared-memory attribute for the current device.  Make that first
+ * call with the right device current and outside any stream capture.
+ *
+ * All calls on a GPU share the one array, which keeps the previous call's
+ * contents; the entry point re-initialises what must start from zero.  Two
+ * calls whose kernels could overlap on the same GPU (different streams,
+ * threads or processes sharing a context) race on it: serialise them.  The
+ * kernel also needs the whole GPU (one cooperative CTA per SM). */
+#define D3_NOALLOC_SCRATCH_BYTES (8u << 20)
+int32_t d3_decode_step_noalloc(const d3_config *cfg, const d3_weights *weights, void *kv_dev,
+                               int32_t slot, int32_t pos, int32_t token, int32_t gen_index,
+                               double alpha, float *logits_dev, void *cuda_stream);
+
 int32_t d3_slot_pos(const d3_model *m, int32_t slot); /* tokens cached; D3_ESTATE if never prefilled */
 int32_t d3_reset_slot(d3_model *m, int32_t slot);
 int32_t d3_sync(d3_model *m); /* wait for the stream; returns a deferred device status */

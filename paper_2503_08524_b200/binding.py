@@ -23,7 +23,7 @@ EXEC_AUTO, EXEC_KERNELS = 0, 1
 
 EXPORTS = ("d3_depth", "d3_schedule", "d3_workspace_bytes", "d3_load", "d3_prefill",
            "d3_decode_step", "d3_argmax", "d3_read_schedule", "d3_read_hidden", "d3_read_kv",
-           "d3_set_exec", "d3_profile", "d3_read_profile", "d3_profile_name", "d3_slot_pos", "d3_reset_slot", "d3_sync", "d3_free", "d3_strerror")
+           "d3_set_exec", "d3_profile", "d3_read_profile", "d3_profile_name", "d3_decode_step_noalloc", "d3_slot_pos", "d3_reset_slot", "d3_sync", "d3_free", "d3_strerror")
 
 
 class Config(C.Structure):
@@ -75,6 +75,8 @@ def _load() -> C.CDLL:
     lib.d3_read_profile.argtypes = [P, P, P]
     lib.d3_profile_name.argtypes = [I32]
     lib.d3_profile_name.restype = C.c_char_p
+    lib.d3_decode_step_noalloc.argtypes = [C.POINTER(Config), C.POINTER(Weights), P, I32, I32, I32, I32,
+                                           C.c_double, P, P]
     lib.d3_slot_pos.argtypes = [P, I32]
     lib.d3_reset_slot.argtypes = [P, I32]
     lib.d3_sync.argtypes = [P]
@@ -130,6 +132,28 @@ def d3_workspace_bytes(cfg: Config):
 
 def _ptrs(tensors: List[torch.Tensor]):
     return (C.c_void_p * len(tensors))(*[t.data_ptr() for t in tensors])
+
+
+NOALLOC_SCRATCH_BYTES = 8 << 20
+
+
+def d3_decode_step_noalloc(cfg: Config, weights: Dict[str, object], kv: torch.Tensor, slot: int, pos: int,
+                           token: int, gen_index: int, alpha: float, logits: torch.Tensor,
+                           stream: Optional[torch.cuda.Stream] = None) -> int:
+    """One batch-1 decode step on the library's built-in scratch array (see
+    include/d3.h).  Every tensor is the caller's; nothing is allocated here.
+    Returns the library's status code instead of raising, so that callers can
+    test the refusals."""
+    arrays = {k: _ptrs(weights[k]) for k in ("attn_norm", "wqkv", "wo", "mlp_norm", "w_gate", "w_up",
+                                             "w_down")}
+    ws = Weights(weights["embed"].data_ptr(), weights["lm_head"].data_ptr(),
+                 weights["final_norm"].data_ptr(),
+                 *[C.cast(arrays[k], _PP) for k in ("attn_norm", "wqkv", "wo", "mlp_norm", "w_gate",
+                                                    "w_up", "w_down")])
+    st = stream if stream is not None else torch.cuda.current_stream(kv.device)
+    return int(LIB.d3_decode_step_noalloc(C.byref(cfg), C.byref(ws), kv.data_ptr(), slot, pos, token,
+                                          gen_index, float(alpha), logits.data_ptr(),
+                                          C.c_void_p(st.cuda_stream)))
 
 
 class D3Model:

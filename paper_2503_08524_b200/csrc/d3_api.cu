@@ -36,7 +36,7 @@ Layout make_layout(const d3_config &c) {
   return y;
 }
 
-static bool config_ok(const d3_config *c) {
+bool config_ok(const d3_config *c) {
   if (!c || c->struct_size != sizeof(d3_config)) return false;
   if (c->n_layers < 1 || c->n_layers > D3_MAX_LAYERS) return false;
   if (c->d_model < 8 || c->d_model % 8) return false;
@@ -60,7 +60,7 @@ static int32_t depth_host(int32_t L, double alpha, int64_t i) {
 }
 
 // thr[n] = smallest i with floor(L alpha^i) < n (n = 1..L); INT32_MAX if none.
-static void thresholds(int32_t L, double alpha, int32_t *thr) {
+void thresholds(int32_t L, double alpha, int32_t *thr) {
   thr[0] = 0;
   const int64_t imax = 0x7ffffffe;
   for (int n = 1; n <= L; ++n) {

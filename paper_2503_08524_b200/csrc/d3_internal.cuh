@@ -110,6 +110,9 @@ struct Layout {
 };
 
 Layout make_layout(const d3_config &c);
+bool config_ok(const d3_config *c);
+// thr[n] = smallest i with floor(L alpha^i) < n, n = 1..L (INT32_MAX if none); thr[0] = 0
+void thresholds(int32_t L, double alpha, int32_t *thr);
 
 // launchers (each enqueues on `st`; returns the number of kernels launched)
 int launch_rope_table(float2 *table, int max_seq, int dh, float base, cudaStream_t st);
