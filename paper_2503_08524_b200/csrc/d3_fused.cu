@@ -1,10 +1,12 @@
 // Batch-1 decode step as ONE persistent cooperative kernel (sm_100a).
 //
-// One CTA per SM.  Warp 8 is the producer: it streams the CTA's share of every
-// weight matrix (and of the static part of the KV cache) through a
+// One CTA per SM.  Warps 8-11 are producers: they stream the CTA's share of
+// every weight matrix (and of the static part of the KV cache) through a
 // shared-memory ring with bulk asynchronous copies (cp.async.bulk + mbarrier
-// transaction counts).  It never waits for the computation, so HBM stays busy
-// across phase boundaries: weights do not depend on activations.  Each ring
+// transaction counts), stage s issued by producer s mod 4 (one warp alone cannot
+// turn stages around fast enough: ~300 ns per stage of barrier traffic).  They
+// never wait for the computation, so HBM stays busy across phase boundaries:
+// weights do not depend on activations.  Each ring
 // stage is consumed by ONE of the warps 0-7 (stage s of a phase by warp s mod 8),
 // so the warps work on eight stages at a time and never synchronise inside a
 // projection.  Phases of a block (RMSNorm+QKV+RoPE+KV append | attention |
@@ -12,24 +14,13 @@
 // grid barriers on a global counter; only the small fp32 activations cross them
 // (through L2, read with ld.global.cg).
 //
-// A ring stage holds eight weight-row segments of 1024 bf16 (a "row group" x
-// k-chunk; rows 2112 bytes apart so that the fragment loads below do not
-// collide on banks), or 8 KB of K plus 8 KB of V for one KV head.  Row groups
-// are issued eight at a time, k-chunk major, so that warp w keeps the running
-// sums of group w in registers across the k-chunks and finishes the group
-// alone (epilogue included).
-//
-// The dot products run on the tensor cores (mma.sync m16n8k16, bf16 x bf16 ->
-// fp32) purely to cut the instruction count: widening and multiplying 8192
-// weights per stage on the FP32 pipe costs ~1000 warp-instructions and made the
-// consumer, not HBM, the bottleneck (see profiles/).  The MMA's 8-wide operand
-// is the eight weight rows; its 16-high operand holds the activation vector
-// split into two bf16 terms, x = hi + lo with hi = bf16(x), lo = bf16(x - hi),
-// whose partial sums are added in fp32, so the activation keeps ~16 mantissa
-// bits (the weights themselves are bf16).  A lane loads 8 consecutive k of its
-// weight row and of its activation term with one 128-bit shared load each and
-// feeds two MMAs; the order of k inside an MMA is a private permutation that
-// both operands share.
+// A ring stage is 16 KB: four weight-row segments of 2048 bf16 (a "row group" x
+// k-chunk), or 8 KB of K plus 8 KB of V for one KV head.  Row groups are issued
+// eight at a time, k-chunk major, so that warp w keeps the four running sums of
+// group w in registers across the k-chunks and finishes the group alone
+// (shuffle reduction + epilogue).  A lane owns 8 consecutive k of every
+// 256-element block, so the activation costs two shared loads per four weight
+// loads.
 //
 // Every wait (mbarrier, release counter, grid barrier) is bounded in time; on
 // expiry the kernel raises D3_ETIMEOUT in the schedule's status word and enters
@@ -45,12 +36,10 @@ namespace d3 {
 namespace {
 
 constexpr int kConsumers = 256;
-constexpr int kFusedThreads = 288;
-constexpr int kChunk = 1024;          // weight elements of one row segment
-constexpr int kGroupRows = 8;         // weight rows of one ring stage
-constexpr int kRowStride = kChunk * 2 + 64;            // bytes between row segments in a stage
-constexpr int kStageBytes = kGroupRows * kRowStride;   // 16896
-constexpr int kKvHalf = 8192;         // bytes of K (and of V) in an attention stage
+constexpr int kProducerWarps = 4;      // each issues the stages s with s mod 4 == its index
+constexpr int kFusedThreads = kConsumers + 32 * kProducerWarps;
+constexpr int kStageBytes = 16384;
+constexpr int kChunk = 2048;          // weight elements of one row segment
 constexpr int kMaxStages = 14;
 constexpr int kMaxGQ = 4;
 
@@ -167,37 +156,35 @@ __device__ __forceinline__ Phase make_phase(const FusedParams &p, int kind, int 
   ph.kind = kind;
   ph.W2 = nullptr;
   const Dims &dm = p.dm;
-  if (kind == PH_QKV) { ph.W = p.layers[layer].wqkv; ph.K = dm.d; ph.R = dm.qkv_rows; ph.groups = dm.qkv_rows / 8; }
-  else if (kind == PH_OPROJ) { ph.W = p.layers[layer].wo; ph.K = dm.Hq * dm.dh; ph.R = dm.d; ph.groups = dm.d / 8; }
-  else if (kind == PH_GATEUP) { ph.W = p.layers[layer].w_gate; ph.W2 = p.layers[layer].w_up; ph.K = dm.d; ph.R = dm.f; ph.groups = dm.f / 4; }
-  else if (kind == PH_DOWN) { ph.W = p.layers[layer].w_down; ph.K = dm.f; ph.R = dm.d; ph.groups = dm.d / 8; }
-  else { ph.W = p.lm_head; ph.K = dm.d; ph.R = dm.V; ph.groups = (dm.V + 7) / 8; }
+  if (kind == PH_QKV) { ph.W = p.layers[layer].wqkv; ph.K = dm.d; ph.R = dm.qkv_rows; ph.groups = dm.qkv_rows / 4; }
+  else if (kind == PH_OPROJ) { ph.W = p.layers[layer].wo; ph.K = dm.Hq * dm.dh; ph.R = dm.d; ph.groups = dm.d / 4; }
+  else if (kind == PH_GATEUP) { ph.W = p.layers[layer].w_gate; ph.W2 = p.layers[layer].w_up; ph.K = dm.d; ph.R = dm.f; ph.groups = dm.f / 2; }
+  else if (kind == PH_DOWN) { ph.W = p.layers[layer].w_down; ph.K = dm.f; ph.R = dm.d; ph.groups = dm.d / 4; }
+  else { ph.W = p.lm_head; ph.K = dm.d; ph.R = dm.V; ph.groups = (dm.V + 3) / 4; }
   split_range(ph.groups, cta, ncta, ph.g0, ph.g1);
   ph.nkc = (ph.K + kChunk - 1) / kChunk;
   return ph;
 }
 
-// pointer of weight row n (0..7) of group g (rows beyond R are clamped)
-//   QKV, q/k heads: four rotary pairs: rows jj..jj+3 and their partners jj+half..
-//   gate/up: four gate rows and the four up rows of the same outputs
-__device__ __forceinline__ const bf16 *group_row(const Phase &ph, const Dims &dm, int g, int n) {
+// pointer of weight row j (0..3) of group g (rows beyond R are clamped)
+__device__ __forceinline__ const bf16 *group_row(const Phase &ph, const Dims &dm, int g, int j) {
   int r;
   if (ph.kind == PH_QKV) {
-    const int per_head = dm.dh / 8, half = dm.dh / 2;
+    const int per_head = dm.dh / 4, half = dm.dh / 2;
     const int rot_groups = (dm.Hq + dm.Hkv) * per_head;
-    if (g < rot_groups) {
-      const int head = g / per_head, jj = (g % per_head) * 4;
-      r = head * dm.dh + jj + (n & 3) + (n >> 2) * half;
+    if (g < rot_groups) {   // q or k head: two rotary pairs (jj, jj+half), (jj+1, jj+1+half)
+      const int head = g / per_head, jj = (g % per_head) * 2;
+      r = head * dm.dh + jj + (j & 1) + (j >> 1) * half;
     } else {
-      r = (dm.Hq + dm.Hkv) * dm.dh + (g - rot_groups) * 8 + n;
+      r = (dm.Hq + dm.Hkv) * dm.dh + (g - rot_groups) * 4 + j;
     }
   } else if (ph.kind == PH_GATEUP) {
-    r = 4 * g + (n & 3);
+    r = 2 * g + (j & 1);   // rows 0,1: gate; rows 2,3: up
   } else {
-    r = 8 * g + n;
+    r = 4 * g + j;
   }
   if (r >= ph.R) r = ph.R - 1;
-  const bf16 *base = (ph.kind == PH_GATEUP && n >= 4) ? ph.W2 : ph.W;
+  const bf16 *base = (ph.kind == PH_GATEUP && j >= 2) ? ph.W2 : ph.W;
   return base + (size_t)r * ph.K;
 }
 
@@ -214,7 +201,7 @@ struct AttSplit {
 __device__ __forceinline__ AttSplit make_att(const FusedParams &p, int gq, int cta, int ncta) {
   AttSplit a;
   a.gq = gq;
-  a.CH = kKvHalf / (p.dm.dh * 2);
+  a.CH = (kStageBytes / 2) / (p.dm.dh * 2);
   a.nch = p.pos / a.CH + 1;
   a.streams = p.dm.Hkv * ((p.dm.Hq / p.dm.Hkv) / gq);
   a.units = a.streams * a.nch;
@@ -230,46 +217,53 @@ __device__ __forceinline__ int cta_of_unit(int u, int units, int ncta) {
   return c;
 }
 
-// ---- producer (all 32 lanes of warp 8 run it) -----------------------------------
+// ---- producers (all 32 lanes of each producer warp run this) ----------------------
 struct Producer {
   const Ctx &c;
-  uint32_t s;   // stages issued so far
+  uint32_t s;     // stages of the step enumerated so far (every producer counts them all)
+  uint32_t pid;   // this warp issues the stages with s % kProducerWarps == pid
   bool ok;
-  __device__ Producer(const Ctx &cc) : c(cc), s(0), ok(true) {}
+  __device__ Producer(const Ctx &cc, uint32_t id) : c(cc), s(0), pid(id), ok(true) {}
+  __device__ __forceinline__ bool mine() const { return s % (uint32_t)kProducerWarps == pid; }
+  // Wait until the slot of stage s is free.  Successive fills of a slot are issued by
+  // different warps, so the release counter (not the parity alone) says which fill
+  // was consumed; the mbarrier wait that follows orders the consumers' reads before
+  // the copy that overwrites them.
   __device__ __forceinline__ bool acquire(uint32_t &slot) {
     const uint32_t ns = (uint32_t)c.p->n_stages;
     slot = s % ns;
-    if (s >= ns) {
-      if (!wait_bar(c, smem_u32(&c.empty[slot]), ((s / ns) - 1u) & 1u)) { ok = false; return false; }
+    const uint32_t fill = s / ns;
+    if (fill > 0) {
+      if (c.released[slot] < fill && !*c.abort_flag) {
+        const uint64_t t0 = now_ns();
+        for (uint32_t it = 1; c.released[slot] < fill && !*c.abort_flag; ++it)
+          if ((it & 63u) == 0u && now_ns() - t0 > c.p->wait_ns) raise_timeout(c);
+      }
+      if (!wait_bar(c, smem_u32(&c.empty[slot]), (fill - 1u) & 1u)) { ok = false; return false; }
     }
     return true;
   }
-  // Lane 4w+j holds the pointers of rows j and j+4 of group w of the current batch
-  // of eight groups; the four lanes of a group issue its eight copies.
+  // Lane 4w+j holds the pointer of row j of group w of the current batch of eight
+  // groups; the four lanes of a group issue its copies.
   __device__ void gemv_phase(const Phase &ph) {
     const Dims &dm = c.p->dm;
     const int lane = threadIdx.x & 31, w = lane >> 2, j = lane & 3;
     for (int S0 = ph.g0; S0 < ph.g1 && ok; S0 += 8) {
       const int nw = min(8, ph.g1 - S0);
-      const bf16 *row_a = nullptr, *row_b = nullptr;
-      if (w < nw) {
-        row_a = group_row(ph, dm, S0 + w, j);
-        row_b = group_row(ph, dm, S0 + w, j + 4);
-      }
+      const bf16 *row = (w < nw) ? group_row(ph, dm, S0 + w, j) : nullptr;
       for (int kc = 0; kc < ph.nkc; ++kc) {
         const int kw = min(kChunk, ph.K - kc * kChunk);
-        for (int ww = 0; ww < nw; ++ww) {
+        for (int ww = 0; ww < nw; ++ww, ++s) {
+          if (!mine()) continue;
           uint32_t slot;
           if (!acquire(slot)) return;
           const uint32_t bar = smem_u32(&c.full[slot]);
-          if (lane == ww * 4) mbar_expect_tx(bar, (uint32_t)kGroupRows * (uint32_t)kw * 2u);
-          __syncwarp();
-          if (w == ww) {
-            const uint32_t dst = smem_u32(c.ring + (size_t)slot * kStageBytes);
-            bulk_g2s(dst + j * kRowStride, row_a + (size_t)kc * kChunk, (uint32_t)kw * 2u, bar);
-            bulk_g2s(dst + (j + 4) * kRowStride, row_b + (size_t)kc * kChunk, (uint32_t)kw * 2u, bar);
-          }
-          ++s;
+          // the copies may complete bytes before the expect_tx lands: the phase cannot
+          // end before its one arrival (the expect_tx itself)
+          if (lane == ww * 4) mbar_expect_tx(bar, 4u * (uint32_t)kw * 2u);
+          if (w == ww)
+            bulk_g2s(smem_u32(c.ring + (size_t)slot * kStageBytes) + j * (kChunk * 2),
+                     row + (size_t)kc * kChunk, (uint32_t)kw * 2u, bar);
         }
       }
     }
@@ -283,16 +277,16 @@ struct Producer {
       const int stream = u / a.nch, chunk = u % a.nch;
       if (chunk == a.nch - 1) continue;   // the chunk with the current position: plain loads
       const int kvh = stream / qgroups;
+      if (!mine()) { ++s; continue; }
       uint32_t slot;
       if (!acquire(slot)) return;
       const size_t off = ((((size_t)layer * dm.max_slots + p.slot) * dm.Hkv + kvh) * dm.max_seq +
                           (size_t)chunk * a.CH) * dm.dh;
       const uint32_t bar = smem_u32(&c.full[slot]);
       const uint32_t dst = smem_u32(c.ring + (size_t)slot * kStageBytes);
-      if (lane == 0) mbar_expect_tx(bar, 2u * (uint32_t)kKvHalf);
-      __syncwarp();
-      if (lane == 0) bulk_g2s(dst, p.Kc + off, kKvHalf, bar);
-      if (lane == 1) bulk_g2s(dst + kKvHalf, p.Vc + off, kKvHalf, bar);
+      if (lane == 0) mbar_expect_tx(bar, (uint32_t)kStageBytes);
+      if (lane == 0) bulk_g2s(dst, p.Kc + off, kStageBytes / 2, bar);
+      if (lane == 1) bulk_g2s(dst + kStageBytes / 2, p.Vc + off, kStageBytes / 2, bar);
       ++s;
     }
   }
@@ -312,39 +306,21 @@ __device__ __forceinline__ float block_sum(float v) {
   return t;
 }
 
-// The activation vector of a projection sits in shared memory as two bf16
-// arrays, x = hi + lo (hi = bf16(x), lo = bf16(x - hi)), lo 64 bytes past a
-// multiple of 128 after hi so that the two terms land on different banks.
-__device__ __forceinline__ uint32_t act_lo_offset(int K) {   // bytes from hi to lo
-  return (uint32_t)((K * 2 + 127) / 128 * 128 + 64);
+// position of element k of an activation vector in the permuted shared layout:
+// within each block of 256 elements, element lane*8 + j sits at (j/4)*128 + lane*4 + j%4
+__device__ __forceinline__ int act_index(int k) {
+  return (k & ~255) + ((k & 7) >> 2) * 128 + ((k & 255) >> 3) * 4 + (k & 3);
 }
 
-__device__ __forceinline__ void store_split4(unsigned char *act, uint32_t lo_off, int k, float4 t) {
-  const __nv_bfloat16 h0 = __float2bfloat16_rn(t.x), h1 = __float2bfloat16_rn(t.y);
-  const __nv_bfloat16 h2 = __float2bfloat16_rn(t.z), h3 = __float2bfloat16_rn(t.w);
-  const __nv_bfloat16 l0 = __float2bfloat16_rn(t.x - __bfloat162float(h0));
-  const __nv_bfloat16 l1 = __float2bfloat16_rn(t.y - __bfloat162float(h1));
-  const __nv_bfloat16 l2 = __float2bfloat16_rn(t.z - __bfloat162float(h2));
-  const __nv_bfloat16 l3 = __float2bfloat16_rn(t.w - __bfloat162float(h3));
-  uint2 hv, lv;
-  hv.x = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
-  hv.y = (uint32_t)__bfloat16_as_ushort(h2) | ((uint32_t)__bfloat16_as_ushort(h3) << 16);
-  lv.x = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
-  lv.y = (uint32_t)__bfloat16_as_ushort(l2) | ((uint32_t)__bfloat16_as_ushort(l3) << 16);
-  *reinterpret_cast<uint2 *>(act + (size_t)k * 2) = hv;
-  *reinterpret_cast<uint2 *>(act + lo_off + (size_t)k * 2) = lv;
-}
-
-// act := src (global fp32, length K) split into hi/lo.  With `gain` the vector
-// (K <= 16 * 1024, the model width) is RMS-normalised first: one pass over L2,
-// the values wait in registers for the scale.
+// act := src (global fp32, length K).  With `gain` the vector (K <= 16 * 1024,
+// the model width) is RMS-normalised: one pass over L2, the values wait in
+// registers for the scale.
 __device__ void load_act(const Ctx &c, const float *src, int K, const bf16 *gain) {
   const int tid = threadIdx.x;
-  unsigned char *act = reinterpret_cast<unsigned char *>(c.act);
-  const uint32_t lo_off = act_lo_offset(K);
   if (!gain) {
 #pragma unroll 4
-    for (int k = tid * 4; k < K; k += kConsumers * 4) store_split4(act, lo_off, k, ldcg4(src + k));
+    for (int k = tid * 4; k < K; k += kConsumers * 4)
+      *reinterpret_cast<float4 *>(c.act + act_index(k)) = ldcg4(src + k);
     consumer_sync();
     return;
   }
@@ -368,19 +344,10 @@ __device__ void load_act(const Ctx &c, const float *src, int K, const bf16 *gain
       const uint2 gw = *reinterpret_cast<const uint2 *>(gain + k);
       t.x *= scale * bfl(gw.x); t.y *= scale * bfh(gw.x);
       t.z *= scale * bfl(gw.y); t.w *= scale * bfh(gw.y);
-      store_split4(act, lo_off, k, t);
+      *reinterpret_cast<float4 *>(c.act + act_index(k)) = t;
     }
   }
   consumer_sync();
-}
-
-__device__ __forceinline__ void mma_bf16(float (&d)[4], uint32_t a0, uint32_t a2, uint32_t b0, uint32_t b1) {
-  // rows 8..15 of the 16-high operand (a1, a3) are zero
-  asm volatile(
-      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
-      "{%0,%1,%2,%3};"
-      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
-      : "r"(a0), "r"(0u), "r"(a2), "r"(0u), "r"(b0), "r"(b1));
 }
 
 struct Consumer {
@@ -416,68 +383,59 @@ struct Consumer {
     }
   }
 
-  // One GEMV phase over the activation vector held (split) in c.act.
-  // Lane (g = lane / 4, t = lane % 4) loads k = 8t..8t+7 of every 32-wide step from
-  // weight row g of the stage, and (g < 2) from activation term g; after the last
-  // k-chunk lane t < 4 of term 0 plus lane t + 4 of term 1 hold the outputs of rows
-  // 2t and 2t + 1 of the group.
+  // One GEMV phase over the activation vector held in c.act.
   __device__ void gemv_phase(const Phase &ph, int layer) {
     const Dims &dm = c.p->dm;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
-    const unsigned char *act = reinterpret_cast<const unsigned char *>(c.act);
-    const uint32_t lo_off = act_lo_offset(ph.K);
-    const unsigned char *a_lane = act + (g == 1 ? lo_off : 0u) + t * 16;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     for (int S0 = ph.g0; S0 < ph.g1; S0 += 8) {
       const int nw = min(8, ph.g1 - S0);
       if (warp < nw) {
-        float d0[4] = {0.f, 0.f, 0.f, 0.f}, d1[4] = {0.f, 0.f, 0.f, 0.f};
+        float acc[4] = {0.f, 0.f, 0.f, 0.f};
         const uint32_t first = s + (uint32_t)(S0 - ph.g0) * (uint32_t)ph.nkc + (uint32_t)warp;
         for (int kc = 0; kc < ph.nkc; ++kc) {
           const uint32_t sn = first + (uint32_t)(kc * nw);
           const uint32_t slot = wait_stage(sn);
           const int kw = min(kChunk, ph.K - kc * kChunk);
-          const unsigned char *w_lane = c.ring + (size_t)slot * kStageBytes + g * kRowStride + t * 16;
-          const unsigned char *a_kc = a_lane + (size_t)kc * (kChunk * 2);
-#pragma unroll 4
-          for (int k0 = 0; k0 < kw; k0 += 32) {
-            uint4 wv = make_uint4(0u, 0u, 0u, 0u), av = make_uint4(0u, 0u, 0u, 0u);
-            if (k0 + t * 8 < kw) {
-              wv = *reinterpret_cast<const uint4 *>(w_lane + k0 * 2);
-              if (g < 2) av = *reinterpret_cast<const uint4 *>(a_kc + k0 * 2);
+          const unsigned char *st = c.ring + (size_t)slot * kStageBytes + lane * 16;
+          const float *a = c.act + kc * kChunk + lane * 4;
+#pragma unroll 2
+          for (int b = 0; b < kChunk / 256; ++b) {
+            if (b * 256 + lane * 8 < kw) {
+              const float4 x0 = *reinterpret_cast<const float4 *>(a + b * 256);
+              const float4 x1 = *reinterpret_cast<const float4 *>(a + b * 256 + 128);
+#pragma unroll
+              for (int j = 0; j < 4; ++j) {
+                const uint4 w = *reinterpret_cast<const uint4 *>(st + j * (kChunk * 2) + b * 512);
+                acc[j] += bfl(w.x) * x0.x + bfh(w.x) * x0.y + bfl(w.y) * x0.z + bfh(w.y) * x0.w +
+                          bfl(w.z) * x1.x + bfh(w.z) * x1.y + bfl(w.w) * x1.z + bfh(w.w) * x1.w;
+              }
             }
-            mma_bf16(d0, av.x, av.y, wv.x, wv.y);
-            mma_bf16(d1, av.z, av.w, wv.z, wv.w);
           }
           release_stage(slot, sn);
         }
-        // hi + lo terms: lanes 4..7 (term 1) onto lanes 0..3 (term 0)
-        float y0 = d0[0] + d1[0], y1 = d0[1] + d1[1];
-        y0 += __shfl_down_sync(0xffffffffu, y0, 4);
-        y1 += __shfl_down_sync(0xffffffffu, y1, 4);
-        // rows n and n + 4 of the group pair up (rotary pair, gate with up): lanes 0,1
-        // fetch rows 4..7 from lanes 2,3
-        const float p0 = __shfl_down_sync(0xffffffffu, y0, 2), p1 = __shfl_down_sync(0xffffffffu, y1, 2);
-        if (lane < 4) epilogue(ph, dm, layer, S0 + warp, lane, y0, y1, p0, p1);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) acc[j] += __shfl_xor_sync(0xffffffffu, acc[j], o);
+        }
+        if (lane == 0) epilogue(ph, dm, layer, S0 + warp, acc[0], acc[1], acc[2], acc[3]);
       }
     }
     s += (uint32_t)(ph.g1 - ph.g0) * (uint32_t)ph.nkc;
   }
 
-  // Lane t (0..3) holds y0, y1 = outputs of rows 2t, 2t+1 of group g; lanes 0,1 also
-  // hold p0, p1 = outputs of rows 2t+4, 2t+5.
-  __device__ void epilogue(const Phase &ph, const Dims &dm, int layer, int g, int t, float y0, float y1,
-                           float p0, float p1) {
+  __device__ void epilogue(const Phase &ph, const Dims &dm, int layer, int g, float y0, float y1, float y2,
+                           float y3) {
     const FusedParams &p = *c.p;
     if (ph.kind == PH_QKV) {
-      const int per_head = dm.dh / 8, half = dm.dh / 2;
+      const int per_head = dm.dh / 4, half = dm.dh / 2;
       const int rot_groups = (dm.Hq + dm.Hkv) * per_head;
       const size_t cbase = ((size_t)layer * dm.max_slots + p.slot) * dm.Hkv;
       if (g < rot_groups) {
-        if (t >= 2) return;
-        const int head = g / per_head, jj = (g % per_head) * 4 + 2 * t;
+        const int head = g / per_head, jj = (g % per_head) * 2;
         const float2 cs0 = p.rope[(size_t)p.pos * half + jj], cs1 = p.rope[(size_t)p.pos * half + jj + 1];
-        const float a0 = y0 * cs0.x - p0 * cs0.y, b0 = y0 * cs0.y + p0 * cs0.x;
-        const float a1 = y1 * cs1.x - p1 * cs1.y, b1 = y1 * cs1.y + p1 * cs1.x;
+        const float a0 = y0 * cs0.x - y2 * cs0.y, b0 = y0 * cs0.y + y2 * cs0.x;
+        const float a1 = y1 * cs1.x - y3 * cs1.y, b1 = y1 * cs1.y + y3 * cs1.x;
         if (head < dm.Hq) {
           float *q = p.qkv + head * dm.dh;
           q[jj] = a0; q[jj + 1] = a1; q[jj + half] = b0; q[jj + half + 1] = b1;
@@ -487,22 +445,24 @@ struct Consumer {
           dst[jj + half] = __float2bfloat16_rn(b0); dst[jj + half + 1] = __float2bfloat16_rn(b1);
         }
       } else {
-        const int r = (g - rot_groups) * 8 + 2 * t, h = r / dm.dh, e = r % dm.dh;
+        const int r = (g - rot_groups) * 4, h = r / dm.dh, e = r % dm.dh;
         bf16 *dst = p.Vc + ((cbase + h) * dm.max_seq + p.pos) * dm.dh + e;
         dst[0] = __float2bfloat16_rn(y0); dst[1] = __float2bfloat16_rn(y1);
+        dst[2] = __float2bfloat16_rn(y2); dst[3] = __float2bfloat16_rn(y3);
       }
     } else if (ph.kind == PH_GATEUP) {
-      if (t >= 2) return;
-      p.u[4 * g + 2 * t] = y0 / (1.f + __expf(-y0)) * p0;
-      p.u[4 * g + 2 * t + 1] = y1 / (1.f + __expf(-y1)) * p1;
+      p.u[2 * g] = y0 / (1.f + __expf(-y0)) * y2;
+      p.u[2 * g + 1] = y1 / (1.f + __expf(-y1)) * y3;
     } else if (ph.kind == PH_HEAD) {
-      const int r = 8 * g + 2 * t;
+      const int r = 4 * g;
       if (r < ph.R) p.logits[r] = y0;
       if (r + 1 < ph.R) p.logits[r + 1] = y1;
+      if (r + 2 < ph.R) p.logits[r + 2] = y2;
+      if (r + 3 < ph.R) p.logits[r + 3] = y3;
     } else {   // O-proj / down: residual add on the rows this CTA owns
-      float2 *xp = reinterpret_cast<float2 *>(p.x + 8 * g + 2 * t);
-      float2 v = __ldcg(xp);
-      v.x += y0; v.y += y1;
+      float4 *xp = reinterpret_cast<float4 *>(p.x + 4 * g);
+      float4 v = __ldcg(xp);
+      v.x += y0; v.y += y1; v.z += y2; v.w += y3;
       *xp = v;
     }
   }
@@ -571,7 +531,7 @@ struct Consumer {
             }
           } else {
             const unsigned char *ks = c.ring + (size_t)slot * kStageBytes + ((size_t)i * DH + part * EPL) * 2;
-            const unsigned char *vs = ks + kKvHalf;
+            const unsigned char *vs = ks + kStageBytes / 2;
 #pragma unroll
             for (int e = 0; e < EPL; e += 4) {
               const uint2 kw = *reinterpret_cast<const uint2 *>(ks + e * 2);
@@ -733,9 +693,9 @@ __global__ void __launch_bounds__(kFusedThreads, 1) k_step_b1(const __grid_const
 
   const AttSplit att = make_att(p, GQ, c.cta, c.ncta);
 
-  if (warp == 8) {
-    // ------------------------------------------------------------ producer
-    Producer pr(c);
+  if (warp >= 8) {
+    // ------------------------------------------------------------ producers
+    Producer pr(c, (uint32_t)(warp - 8));
     for (int l = 0; l < L && pr.ok; ++l) {
       if (lo <= l && l < hi) continue;
       pr.gemv_phase(make_phase(p, PH_QKV, l, c.cta, c.ncta));
@@ -750,6 +710,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) k_step_b1(const __grid_const
       const uint32_t ns = (uint32_t)p.n_stages;
       const uint32_t first = pr.s > ns ? pr.s - ns : 0;
       for (uint32_t s = first; s < pr.s; ++s) {
+        if (s % (uint32_t)kProducerWarps != pr.pid) continue;
         const uint32_t bar = smem_u32(&s_full[s % ns]);
         const uint64_t t0 = now_ns();
         while (!mbar_try_wait(bar, (s / ns) & 1u) && now_ns() - t0 < p.wait_ns) {}
@@ -867,14 +828,12 @@ static bool try_plan(FusedPlan &pl, const d3_config &c) {
   cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
   cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev);
   if (!coop || sms < 1) return false;
-  int kmax = c.d_model;
-  if (c.d_ffn > kmax) kmax = c.d_ffn;
-  if (c.n_q_heads * c.head_dim > kmax) kmax = c.n_q_heads * c.head_dim;
-  // hi and lo bf16 arrays of the widest activation vector, or the attention merge scratch
-  int need = (2 * ((kmax * 2 + 127) / 128 * 128 + 64) + 3) / 4;
+  int need = c.d_model;
+  if (c.d_ffn > need) need = c.d_ffn;
+  if (c.n_q_heads * c.head_dim > need) need = c.n_q_heads * c.head_dim;
+  need = (need + kChunk - 1) / kChunk * kChunk;
   const int att_need = 8 * kMaxGQ * (128 + 2) + kFusedMaxCtas * (1 + 2 * kMaxGQ);
-  if (need < att_need) need = att_need;
-  need = (need + 255) / 256 * 256;
+  if (need < att_need) need = (att_need + kChunk - 1) / kChunk * kChunk;
   const int reserve = 4096;   // static shared memory of the kernel and slack
   int stages = (optin - reserve - need * 4) / kStageBytes;
   if (stages > kMaxStages) stages = kMaxStages;
@@ -905,7 +864,7 @@ int fused_plan(const d3_config &c, int *grid, int *n_stages, int *act_floats, si
   const int G = c.n_q_heads / c.n_kv_heads;
   const int gq = (G % 4 == 0) ? 4 : (G % 2 == 0) ? 2 : 1;
   bool ok = false;
-  if (c.d_model <= 16 * 1024) {
+  if (c.vocab % 4 == 0 && c.d_model <= 16 * 1024) {
     if (c.head_dim == 128 && gq == 1) ok = try_plan<128, 1>(pl, c);
     else if (c.head_dim == 128 && gq == 4) ok = try_plan<128, 4>(pl, c);
     else if (c.head_dim == 64 && gq == 1) ok = try_plan<64, 1>(pl, c);
