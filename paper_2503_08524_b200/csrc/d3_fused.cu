@@ -42,6 +42,7 @@ constexpr int kStageBytes = 16384;
 constexpr int kChunk = 2048;          // weight elements of one row segment
 constexpr int kMaxStages = 14;
 constexpr int kMaxGQ = 4;
+constexpr int kMaxOwnRows = 1024;     // residual-stream rows one CTA may own (d / #CTAs, rounded up)
 
 enum PhaseKind { PH_QKV = 0, PH_OPROJ, PH_GATEUP, PH_DOWN, PH_HEAD };
 
@@ -92,6 +93,8 @@ struct Ctx {
   uint64_t *full, *empty;
   volatile uint32_t *released;   // per slot: fills consumed so far
   volatile int *abort_flag;
+  float *x_own;      // this CTA's rows of the residual stream (the rows its O-proj/down groups own)
+  float2 *rope_row;  // (cos, sin) of the step's position
   int cta, ncta;
 };
 
@@ -118,11 +121,13 @@ __device__ __forceinline__ bool wait_bar(const Ctx &c, uint32_t bar, uint32_t pa
 }
 
 // Grid barrier number `idx` (1-based) among the consumer threads of all CTAs.
+// bar.sync orders the CTA's writes before thread 0; its release-add publishes them
+// at GPU scope; the acquire-load that sees the full count orders the other CTAs'
+// writes before everything after the second bar.sync.
 __device__ __forceinline__ void grid_barrier(const Ctx &c, unsigned idx) {
   consumer_sync();
   if (threadIdx.x == 0) {
-    __threadfence();
-    atomicAdd(c.p->bar_counter, 1u);
+    asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(c.p->bar_counter) : "memory");
     const unsigned target = idx * (unsigned)c.ncta;
     const uint64_t t0 = now_ns();
     for (uint32_t it = 1; !*c.abort_flag; ++it) {
@@ -131,7 +136,6 @@ __device__ __forceinline__ void grid_barrier(const Ctx &c, unsigned idx) {
       if (v >= target) break;
       if ((it & 15u) == 0u && now_ns() - t0 > c.p->wait_ns) raise_timeout(c);
     }
-    __threadfence();
   }
   consumer_sync();
 }
@@ -312,23 +316,37 @@ __device__ __forceinline__ int act_index(int k) {
   return (k & ~255) + ((k & 7) >> 2) * 128 + ((k & 255) >> 3) * 4 + (k & 3);
 }
 
-// act := src (global fp32, length K).  With `gain` the vector (K <= 16 * 1024,
-// the model width) is RMS-normalised: one pass over L2, the values wait in
-// registers for the scale.
-__device__ void load_act(const Ctx &c, const float *src, int K, const bf16 *gain) {
-  const int tid = threadIdx.x;
-  if (!gain) {
-#pragma unroll 4
-    for (int k = tid * 4; k < K; k += kConsumers * 4)
-      *reinterpret_cast<float4 *>(c.act + act_index(k)) = ldcg4(src + k);
-    consumer_sync();
-    return;
+// RMSNorm gains of the next normalised load, fetched into registers before the
+// grid barrier (they are weights: nothing to wait for), so that the load after the
+// barrier costs one L2 round trip only.
+struct GainRegs {
+  static constexpr int kMaxIt = 16;   // 16 * 1024 elements
+  uint2 g[kMaxIt];
+};
+__device__ __forceinline__ void prefetch_gain(GainRegs &gr, const bf16 *gain, int K) {
+#pragma unroll
+  for (int it = 0; it < GainRegs::kMaxIt; ++it) {
+    const int k = it * (kConsumers * 4) + threadIdx.x * 4;
+    if (k < K) gr.g[it] = *reinterpret_cast<const uint2 *>(gain + k);
   }
-  constexpr int kMaxIt = 16;   // 16 * 1024 floats
-  float4 v[kMaxIt];
+}
+
+// act := src (global fp32, length K), no normalisation
+__device__ void load_act_plain(const Ctx &c, const float *src, int K) {
+#pragma unroll 4
+  for (int k = threadIdx.x * 4; k < K; k += kConsumers * 4)
+    *reinterpret_cast<float4 *>(c.act + act_index(k)) = ldcg4(src + k);
+  consumer_sync();
+}
+
+// act := RMSNorm(src) * gain (K <= 16 * 1024, the model width): one pass over L2,
+// the values wait in registers for the scale
+__device__ void load_act_norm(const Ctx &c, const float *src, int K, const GainRegs &gr) {
+  const int tid = threadIdx.x;
+  float4 v[GainRegs::kMaxIt];
   float ss = 0.f;
 #pragma unroll
-  for (int it = 0; it < kMaxIt; ++it) {
+  for (int it = 0; it < GainRegs::kMaxIt; ++it) {
     const int k = it * (kConsumers * 4) + tid * 4;
     if (k < K) {
       v[it] = ldcg4(src + k);
@@ -337,11 +355,11 @@ __device__ void load_act(const Ctx &c, const float *src, int K, const bf16 *gain
   }
   const float scale = rsqrtf(block_sum(ss) / (float)K + c.p->eps);
 #pragma unroll
-  for (int it = 0; it < kMaxIt; ++it) {
+  for (int it = 0; it < GainRegs::kMaxIt; ++it) {
     const int k = it * (kConsumers * 4) + tid * 4;
     if (k < K) {
       float4 t = v[it];
-      const uint2 gw = *reinterpret_cast<const uint2 *>(gain + k);
+      const uint2 gw = gr.g[it];
       t.x *= scale * bfl(gw.x); t.y *= scale * bfh(gw.x);
       t.z *= scale * bfl(gw.y); t.w *= scale * bfh(gw.y);
       *reinterpret_cast<float4 *>(c.act + act_index(k)) = t;
@@ -433,7 +451,7 @@ struct Consumer {
       const size_t cbase = ((size_t)layer * dm.max_slots + p.slot) * dm.Hkv;
       if (g < rot_groups) {
         const int head = g / per_head, jj = (g % per_head) * 2;
-        const float2 cs0 = p.rope[(size_t)p.pos * half + jj], cs1 = p.rope[(size_t)p.pos * half + jj + 1];
+        const float2 cs0 = c.rope_row[jj], cs1 = c.rope_row[jj + 1];
         const float a0 = y0 * cs0.x - y2 * cs0.y, b0 = y0 * cs0.y + y2 * cs0.x;
         const float a1 = y1 * cs1.x - y3 * cs1.y, b1 = y1 * cs1.y + y3 * cs1.x;
         if (head < dm.Hq) {
@@ -459,11 +477,13 @@ struct Consumer {
       if (r + 1 < ph.R) p.logits[r + 1] = y1;
       if (r + 2 < ph.R) p.logits[r + 2] = y2;
       if (r + 3 < ph.R) p.logits[r + 3] = y3;
-    } else {   // O-proj / down: residual add on the rows this CTA owns
-      float4 *xp = reinterpret_cast<float4 *>(p.x + 4 * g);
-      float4 v = __ldcg(xp);
+    } else {   // O-proj / down: residual add on the rows this CTA owns (its own copy
+               // is current: no other CTA ever writes them), published for the others
+      float4 *own = reinterpret_cast<float4 *>(c.x_own + 4 * (g - ph.g0));
+      float4 v = *own;
       v.x += y0; v.y += y1; v.z += y2; v.w += y3;
-      *xp = v;
+      *own = v;
+      *reinterpret_cast<float4 *>(p.x + 4 * g) = v;
     }
   }
 
@@ -661,6 +681,8 @@ __global__ void __launch_bounds__(kFusedThreads, 1) k_step_b1(const __grid_const
   __shared__ __align__(8) uint64_t s_full[kMaxStages], s_empty[kMaxStages];
   __shared__ uint32_t s_released[kMaxStages];
   __shared__ int s_abort;
+  __shared__ __align__(16) float s_x_own[kMaxOwnRows];
+  __shared__ float2 s_rope[64];
   const int tid = threadIdx.x, warp = tid >> 5;
   Ctx c;
   c.p = &p;
@@ -669,6 +691,8 @@ __global__ void __launch_bounds__(kFusedThreads, 1) k_step_b1(const __grid_const
   c.full = s_full; c.empty = s_empty;
   c.released = s_released;
   c.abort_flag = &s_abort;
+  c.x_own = s_x_own;
+  c.rope_row = s_rope;
   c.cta = blockIdx.x; c.ncta = gridDim.x;
   if (tid == 0) {
     s_abort = 0;
@@ -728,15 +752,22 @@ __global__ void __launch_bounds__(kFusedThreads, 1) k_step_b1(const __grid_const
     for (int l = 0; l < L; ++l) s->m[l] = (lo <= l && l < hi) ? 0 : 1;
     s->rows_layers = n; s->layers_touched = n;
   }
-  // embedding row -> residual stream (CTA 0 publishes it)
+  // embedding row -> residual stream: CTA 0 publishes it, every CTA keeps its own rows
   const Dims &dm = p.dm;
+  const bf16 *emb = p.embed + (size_t)tok * dm.d;
   if (c.cta == 0) {
-    const bf16 *e = p.embed + (size_t)tok * dm.d;
     for (int k = tid * 8; k < dm.d; k += kConsumers * 8) {
-      const uint4 w = *reinterpret_cast<const uint4 *>(e + k);
+      const uint4 w = *reinterpret_cast<const uint4 *>(emb + k);
       *reinterpret_cast<float4 *>(p.x + k) = make_float4(bfl(w.x), bfh(w.x), bfl(w.y), bfh(w.y));
       *reinterpret_cast<float4 *>(p.x + k + 4) = make_float4(bfl(w.z), bfh(w.z), bfl(w.w), bfh(w.w));
     }
+  }
+  {
+    int og0, og1;
+    split_range(dm.d / 4, c.cta, c.ncta, og0, og1);
+    for (int i = tid; i < (og1 - og0) * 4; i += kConsumers)
+      s_x_own[i] = __bfloat162float(emb[og0 * 4 + i]);
+    for (int i = tid; i < dm.dh / 2; i += kConsumers) s_rope[i] = p.rope[(size_t)p.pos * (dm.dh / 2) + i];
   }
   Consumer cs(c);
   unsigned bidx = 0, ordinal = 0;
@@ -750,11 +781,17 @@ __global__ void __launch_bounds__(kFusedThreads, 1) k_step_b1(const __grid_const
       t_prev = t;
     }
   };
+  // first executed block (or L when the row runs none)
+  int l = 0;
+  while (l < L && lo <= l && l < hi) ++l;
+  GainRegs gr;
+  prefetch_gain(gr, l < L ? p.layers[l].attn_norm : p.final_norm, dm.d);
   grid_barrier(c, ++bidx);
   tick(0);
-  for (int l = 0; l < L; ++l) {
-    if (lo <= l && l < hi) continue;   // dropped block: the hidden state passes through
-    load_act(c, p.x, dm.d, p.layers[l].attn_norm);
+  while (l < L) {
+    int next = l + 1;   // dropped blocks: the hidden state passes through
+    while (next < L && lo <= next && next < hi) ++next;
+    load_act_norm(c, p.x, dm.d, gr);
     tick(1);
     cs.gemv_phase(make_phase(p, PH_QKV, l, c.cta, c.ncta), l);
     tick(2);
@@ -764,24 +801,27 @@ __global__ void __launch_bounds__(kFusedThreads, 1) k_step_b1(const __grid_const
     tick(4);
     grid_barrier(c, ++bidx);
     tick(3);
-    load_act(c, p.attn_out, dm.Hq * dm.dh, nullptr);
+    load_act_plain(c, p.attn_out, dm.Hq * dm.dh);
     tick(1);
     cs.gemv_phase(make_phase(p, PH_OPROJ, l, c.cta, c.ncta), l);
     tick(5);
+    prefetch_gain(gr, p.layers[l].mlp_norm, dm.d);
     grid_barrier(c, ++bidx);
     tick(3);
-    load_act(c, p.x, dm.d, p.layers[l].mlp_norm);
+    load_act_norm(c, p.x, dm.d, gr);
     tick(1);
     cs.gemv_phase(make_phase(p, PH_GATEUP, l, c.cta, c.ncta), l);
     tick(6);
     grid_barrier(c, ++bidx);
     tick(3);
-    load_act(c, p.u, dm.f, nullptr);
+    load_act_plain(c, p.u, dm.f);
     tick(1);
     cs.gemv_phase(make_phase(p, PH_DOWN, l, c.cta, c.ncta), l);
     tick(7);
+    prefetch_gain(gr, next < L ? p.layers[next].attn_norm : p.final_norm, dm.d);
     grid_barrier(c, ++bidx);
     tick(3);
+    l = next;
   }
   // KV fill by copy for the dropped blocks: CTA j takes block lo + j, lo + j + ncta, ...
   if (p.kv_fill == D3_FILL_COPY) {
@@ -804,7 +844,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) k_step_b1(const __grid_const
     }
   }
   if (p.logits) {
-    load_act(c, p.x, dm.d, p.final_norm);
+    load_act_norm(c, p.x, dm.d, gr);
     cs.gemv_phase(make_phase(p, PH_HEAD, 0, c.cta, c.ncta), 0);
   }
   tick(8);
@@ -828,13 +868,15 @@ static bool try_plan(FusedPlan &pl, const d3_config &c) {
   cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
   cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev);
   if (!coop || sms < 1) return false;
+  const int ctas = sms < kFusedMaxCtas ? sms : kFusedMaxCtas;
+  if ((c.d_model / 4 / ctas + 2) * 4 > kMaxOwnRows) return false;   // the CTA's own rows of x
   int need = c.d_model;
   if (c.d_ffn > need) need = c.d_ffn;
   if (c.n_q_heads * c.head_dim > need) need = c.n_q_heads * c.head_dim;
   need = (need + kChunk - 1) / kChunk * kChunk;
   const int att_need = 8 * kMaxGQ * (128 + 2) + kFusedMaxCtas * (1 + 2 * kMaxGQ);
   if (need < att_need) need = (att_need + kChunk - 1) / kChunk * kChunk;
-  const int reserve = 4096;   // static shared memory of the kernel and slack
+  const int reserve = 8192;   // static shared memory of the kernel and slack
   int stages = (optin - reserve - need * 4) / kStageBytes;
   if (stages > kMaxStages) stages = kMaxStages;
   if (const char *env = getenv("D3_FUSED_STAGES")) {   // tuning knob: a shallower ring
