@@ -318,12 +318,14 @@ __device__ __forceinline__ int act_index(int k) {
 
 // RMSNorm gains of the next normalised load, fetched into registers before the
 // grid barrier (they are weights: nothing to wait for), so that the load after the
-// barrier costs one L2 round trip only.
+// barrier costs one L2 round trip only.  Widths up to 4096 take this path; wider
+// vectors are normalised in two passes and read their gains in the second.
 struct GainRegs {
-  static constexpr int kMaxIt = 16;   // 16 * 1024 elements
+  static constexpr int kMaxIt = 4;   // 4 * 1024 elements
   uint2 g[kMaxIt];
 };
 __device__ __forceinline__ void prefetch_gain(GainRegs &gr, const bf16 *gain, int K) {
+  if (K > GainRegs::kMaxIt * kConsumers * 4) return;
 #pragma unroll
   for (int it = 0; it < GainRegs::kMaxIt; ++it) {
     const int k = it * (kConsumers * 4) + threadIdx.x * 4;
@@ -339,27 +341,43 @@ __device__ void load_act_plain(const Ctx &c, const float *src, int K) {
   consumer_sync();
 }
 
-// act := RMSNorm(src) * gain (K <= 16 * 1024, the model width): one pass over L2,
-// the values wait in registers for the scale
-__device__ void load_act_norm(const Ctx &c, const float *src, int K, const GainRegs &gr) {
+// act := RMSNorm(src) * gain.  Up to 4096 elements: one pass over L2, the values wait
+// in registers for the scale.  Wider: sum of squares first, then a second pass.
+__device__ void load_act_norm(const Ctx &c, const float *src, int K, const GainRegs &gr, const bf16 *gain) {
   const int tid = threadIdx.x;
-  float4 v[GainRegs::kMaxIt];
-  float ss = 0.f;
+  if (K <= GainRegs::kMaxIt * kConsumers * 4) {
+    float4 v[GainRegs::kMaxIt];
+    float ss = 0.f;
 #pragma unroll
-  for (int it = 0; it < GainRegs::kMaxIt; ++it) {
-    const int k = it * (kConsumers * 4) + tid * 4;
-    if (k < K) {
-      v[it] = ldcg4(src + k);
-      ss += v[it].x * v[it].x + v[it].y * v[it].y + v[it].z * v[it].z + v[it].w * v[it].w;
+    for (int it = 0; it < GainRegs::kMaxIt; ++it) {
+      const int k = it * (kConsumers * 4) + tid * 4;
+      if (k < K) {
+        v[it] = ldcg4(src + k);
+        ss += v[it].x * v[it].x + v[it].y * v[it].y + v[it].z * v[it].z + v[it].w * v[it].w;
+      }
     }
-  }
-  const float scale = rsqrtf(block_sum(ss) / (float)K + c.p->eps);
+    const float scale = rsqrtf(block_sum(ss) / (float)K + c.p->eps);
 #pragma unroll
-  for (int it = 0; it < GainRegs::kMaxIt; ++it) {
-    const int k = it * (kConsumers * 4) + tid * 4;
-    if (k < K) {
-      float4 t = v[it];
-      const uint2 gw = gr.g[it];
+    for (int it = 0; it < GainRegs::kMaxIt; ++it) {
+      const int k = it * (kConsumers * 4) + tid * 4;
+      if (k < K) {
+        float4 t = v[it];
+        const uint2 gw = gr.g[it];
+        t.x *= scale * bfl(gw.x); t.y *= scale * bfh(gw.x);
+        t.z *= scale * bfl(gw.y); t.w *= scale * bfh(gw.y);
+        *reinterpret_cast<float4 *>(c.act + act_index(k)) = t;
+      }
+    }
+  } else {
+    float ss = 0.f;
+    for (int k = tid * 4; k < K; k += kConsumers * 4) {
+      const float4 t = ldcg4(src + k);
+      ss += t.x * t.x + t.y * t.y + t.z * t.z + t.w * t.w;
+    }
+    const float scale = rsqrtf(block_sum(ss) / (float)K + c.p->eps);
+    for (int k = tid * 4; k < K; k += kConsumers * 4) {
+      float4 t = ldcg4(src + k);
+      const uint2 gw = *reinterpret_cast<const uint2 *>(gain + k);
       t.x *= scale * bfl(gw.x); t.y *= scale * bfh(gw.x);
       t.z *= scale * bfl(gw.y); t.w *= scale * bfh(gw.y);
       *reinterpret_cast<float4 *>(c.act + act_index(k)) = t;
@@ -785,13 +803,14 @@ __global__ void __launch_bounds__(kFusedThreads, 1) k_step_b1(const __grid_const
   int l = 0;
   while (l < L && lo <= l && l < hi) ++l;
   GainRegs gr;
-  prefetch_gain(gr, l < L ? p.layers[l].attn_norm : p.final_norm, dm.d);
+  const bf16 *gain = l < L ? p.layers[l].attn_norm : p.final_norm;
+  prefetch_gain(gr, gain, dm.d);
   grid_barrier(c, ++bidx);
   tick(0);
   while (l < L) {
     int next = l + 1;   // dropped blocks: the hidden state passes through
     while (next < L && lo <= next && next < hi) ++next;
-    load_act_norm(c, p.x, dm.d, gr);
+    load_act_norm(c, p.x, dm.d, gr, gain);
     tick(1);
     cs.gemv_phase(make_phase(p, PH_QKV, l, c.cta, c.ncta), l);
     tick(2);
@@ -805,10 +824,11 @@ __global__ void __launch_bounds__(kFusedThreads, 1) k_step_b1(const __grid_const
     tick(1);
     cs.gemv_phase(make_phase(p, PH_OPROJ, l, c.cta, c.ncta), l);
     tick(5);
-    prefetch_gain(gr, p.layers[l].mlp_norm, dm.d);
+    gain = p.layers[l].mlp_norm;
+    prefetch_gain(gr, gain, dm.d);
     grid_barrier(c, ++bidx);
     tick(3);
-    load_act_norm(c, p.x, dm.d, gr);
+    load_act_norm(c, p.x, dm.d, gr, gain);
     tick(1);
     cs.gemv_phase(make_phase(p, PH_GATEUP, l, c.cta, c.ncta), l);
     tick(6);
@@ -818,7 +838,8 @@ __global__ void __launch_bounds__(kFusedThreads, 1) k_step_b1(const __grid_const
     tick(1);
     cs.gemv_phase(make_phase(p, PH_DOWN, l, c.cta, c.ncta), l);
     tick(7);
-    prefetch_gain(gr, next < L ? p.layers[next].attn_norm : p.final_norm, dm.d);
+    gain = next < L ? p.layers[next].attn_norm : p.final_norm;
+    prefetch_gain(gr, gain, dm.d);
     grid_barrier(c, ++bidx);
     tick(3);
     l = next;
@@ -844,7 +865,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) k_step_b1(const __grid_const
     }
   }
   if (p.logits) {
-    load_act_norm(c, p.x, dm.d, gr);
+    load_act_norm(c, p.x, dm.d, gr, gain);
     cs.gemv_phase(make_phase(p, PH_HEAD, 0, c.cta, c.ncta), 0);
   }
   tick(8);
