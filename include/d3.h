@@ -183,6 +183,10 @@ int32_t d3_set_exec(d3_model *m, int32_t mode);
 int32_t d3_profile(d3_model *m, int32_t enable);
 int32_t d3_read_profile(d3_model *m, float *ms, int32_t *launches);
 const char *d3_profile_name(int32_t kind);
+/* The raw per-CTA counters behind the "fused:" figures, without clearing them:
+ * cycles [ctas][phases] int64 (HOST, room for 192 x 16), counts returned in
+ * *ctas and *phases.  Phase order as in d3_profile_name(D3_PROF_FUSED0 + k). */
+int32_t d3_read_fused_phases(d3_model *m, int64_t *cycles, int32_t *ctas, int32_t *phases);
 
 /* One batch-1 decode step that allocates nothing.  (The paper has no
  * counterpart: this entry point exists for the sake of the caller, not of the

@@ -23,7 +23,7 @@ EXEC_AUTO, EXEC_KERNELS = 0, 1
 
 EXPORTS = ("d3_depth", "d3_schedule", "d3_workspace_bytes", "d3_load", "d3_prefill",
            "d3_decode_step", "d3_argmax", "d3_read_schedule", "d3_read_hidden", "d3_read_kv",
-           "d3_set_exec", "d3_profile", "d3_read_profile", "d3_profile_name", "d3_decode_step_noalloc", "d3_slot_pos", "d3_reset_slot", "d3_sync", "d3_free", "d3_strerror")
+           "d3_set_exec", "d3_profile", "d3_read_profile", "d3_profile_name", "d3_read_fused_phases", "d3_decode_step_noalloc", "d3_slot_pos", "d3_reset_slot", "d3_sync", "d3_free", "d3_strerror")
 
 
 class Config(C.Structure):
@@ -73,6 +73,7 @@ def _load() -> C.CDLL:
     lib.d3_set_exec.argtypes = [P, I32]
     lib.d3_profile.argtypes = [P, I32]
     lib.d3_read_profile.argtypes = [P, P, P]
+    lib.d3_read_fused_phases.argtypes = [P, P, P, P]
     lib.d3_profile_name.argtypes = [I32]
     lib.d3_profile_name.restype = C.c_char_p
     lib.d3_decode_step_noalloc.argtypes = [C.POINTER(Config), C.POINTER(Weights), P, I32, I32, I32, I32,
@@ -296,6 +297,15 @@ class D3Model:
             raise D3Error(rc, "d3_read_profile")
         return {LIB.d3_profile_name(k).decode(): {"ms": float(ms[k]), "launches": int(cnt[k])}
                 for k in range(PROF_KINDS) if cnt[k] > 0}
+
+    def d3_read_fused_phases(self) -> np.ndarray:
+        """Per-CTA cycle counters of the single-kernel step's phases, [ctas][phases] (not cleared)."""
+        buf = np.zeros((192, 16), np.int64)
+        nc, nph = C.c_int32(), C.c_int32()
+        rc = LIB.d3_read_fused_phases(self.h, buf.ctypes.data, C.byref(nc), C.byref(nph))
+        if rc != OK:
+            raise D3Error(rc, "d3_read_fused_phases")
+        return buf.reshape(-1)[:nc.value * nph.value].reshape(nc.value, nph.value).copy()
 
     def d3_slot_pos(self, slot: int) -> int:
         return int(LIB.d3_slot_pos(self.h, slot))

@@ -636,6 +636,18 @@ int32_t d3_read_profile(d3_model *m, float *ms, int32_t *launches) {
   return D3_OK;
 }
 
+int32_t d3_read_fused_phases(d3_model *m, int64_t *cycles, int32_t *ctas, int32_t *phases) {
+  if (!m || !cycles || !ctas || !phases) return D3_EINVAL;
+  *ctas = m->fused_ok ? m->fused_grid : 0;
+  *phases = kFusedPhases;
+  if (!m->fused_ok) return D3_OK;
+  if (cudaStreamSynchronize(m->stream) != cudaSuccess) return D3_ECUDA;
+  if (cudaMemcpy(cycles, m->scratch + m->lay.phase, (size_t)m->fused_grid * kFusedPhases * 8,
+                 cudaMemcpyDeviceToHost) != cudaSuccess)
+    return D3_ECUDA;
+  return D3_OK;
+}
+
 const char *d3_profile_name(int32_t kind) {
   return (kind >= 0 && kind < D3_PROF_KINDS) ? kProfNames[kind] : "";
 }

@@ -789,13 +789,19 @@ __global__ void __launch_bounds__(kFusedThreads, 1) k_step_b1(const __grid_const
   }
   Consumer cs(c);
   unsigned bidx = 0, ordinal = 0;
-  // optional phase timer (thread 0 of every CTA): cycles spent up to each phase boundary
+  // optional phase timer (thread 0 of every CTA): cycles spent up to each phase
+  // boundary, summed in registers and written once at the end
   const bool timing = p.phase_cycles != nullptr && tid == 0;
   long long t_prev = clock64();
+  long long t_acc[kFusedPhases];
+#pragma unroll
+  for (int k = 0; k < kFusedPhases; ++k) t_acc[k] = 0;
   auto tick = [&](int k) {
     if (timing) {
       const long long t = clock64();
-      p.phase_cycles[c.cta * kFusedPhases + k] += t - t_prev;
+#pragma unroll
+      for (int q = 0; q < kFusedPhases; ++q)
+        if (q == k) t_acc[q] += t - t_prev;
       t_prev = t;
     }
   };
@@ -869,7 +875,11 @@ __global__ void __launch_bounds__(kFusedThreads, 1) k_step_b1(const __grid_const
     cs.gemv_phase(make_phase(p, PH_HEAD, 0, c.cta, c.ncta), 0);
   }
   tick(8);
-  if (timing) p.phase_cycles[c.cta * kFusedPhases + 9] += cs.ring_wait;
+  if (timing) {
+    t_acc[9] = cs.ring_wait;
+#pragma unroll
+    for (int k = 0; k < kFusedPhases; ++k) p.phase_cycles[c.cta * kFusedPhases + k] += t_acc[k];
+  }
 }
 
 }  // namespace
