@@ -285,6 +285,7 @@ static int32_t run_fused_step(d3_model *m, const StepArgs &a, float *logits_dev,
   fp.part = reinterpret_cast<float *>(m->scratch + m->lay.part_fused);
   fp.logits = logits_dev;
   fp.n_stages = m->fused_stages; fp.act_floats = m->fused_act;
+  fp.l2_window = fused_l2_window();
   fp.wait_ns = 2000000000ull;
   int rc;
   {

@@ -1,12 +1,16 @@
 // Batch-1 decode step as ONE persistent cooperative kernel (sm_100a).
 //
-// One CTA per SM.  Warps 8-11 are producers: they stream the CTA's share of
+// One CTA per SM.  Warps 8-10 are producers: they stream the CTA's share of
 // every weight matrix (and of the static part of the KV cache) through a
 // shared-memory ring with bulk asynchronous copies (cp.async.bulk + mbarrier
-// transaction counts), stage s issued by producer s mod 4 (one warp alone cannot
+// transaction counts), stage s issued by producer s mod 3 (one warp alone cannot
 // turn stages around fast enough: ~300 ns per stage of barrier traffic).  They
-// never wait for the computation, so HBM stays busy across phase boundaries:
-// weights do not depend on activations.  Each ring
+// never wait for the computation: weights do not depend on activations.  Warp 11
+// walks the same sequence of stages further ahead and only asks L2 for them
+// (cp.async.bulk.prefetch.L2): the ring holds ~4 us of HBM time, a phase boundary
+// stalls the consumers for longer (each cross-CTA round trip costs 1-2 us), and
+// with the look-ahead window in L2 HBM keeps streaming through the stall while the
+// ring refills from L2 afterwards.  Each ring
 // stage is consumed by ONE of the warps 0-7 (stage s of a phase by warp s mod 8),
 // so the warps work on eight stages at a time and never synchronise inside a
 // projection.  Phases of a block (RMSNorm+QKV+RoPE+KV append | attention |
@@ -36,8 +40,8 @@ namespace d3 {
 namespace {
 
 constexpr int kConsumers = 256;
-constexpr int kProducerWarps = 4;      // each issues the stages s with s mod 4 == its index
-constexpr int kFusedThreads = kConsumers + 32 * kProducerWarps;
+constexpr int kProducerWarps = 3;      // each issues the stages s with s mod 3 == its index
+constexpr int kFusedThreads = kConsumers + 32 * (kProducerWarps + 1);   // + the L2 prefetcher warp
 constexpr int kStageBytes = 16384;
 constexpr int kChunk = 2048;          // weight elements of one row segment
 constexpr int kMaxStages = 14;
@@ -93,6 +97,7 @@ struct Ctx {
   uint64_t *full, *empty;
   volatile uint32_t *released;   // per slot: fills consumed so far
   volatile int *abort_flag;
+  volatile uint32_t *progress;   // stages issued into the ring so far (producer 0's count)
   float *x_own;      // this CTA's rows of the residual stream (the rows its O-proj/down groups own)
   float2 *rope_row;  // (cos, sin) of the step's position
   int cta, ncta;
@@ -222,13 +227,31 @@ __device__ __forceinline__ int cta_of_unit(int u, int units, int ncta) {
 }
 
 // ---- producers (all 32 lanes of each producer warp run this) ----------------------
+__device__ __forceinline__ void l2_prefetch(const void *src, uint32_t bytes) {
+  asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(bytes) : "memory");
+}
+
 struct Producer {
   const Ctx &c;
   uint32_t s;     // stages of the step enumerated so far (every producer counts them all)
   uint32_t pid;   // this warp issues the stages with s % kProducerWarps == pid
   bool ok;
-  __device__ Producer(const Ctx &cc, uint32_t id) : c(cc), s(0), pid(id), ok(true) {}
-  __device__ __forceinline__ bool mine() const { return s % (uint32_t)kProducerWarps == pid; }
+  bool l2_only;   // the prefetcher: every stage, L2 prefetch only, a bounded distance ahead
+  __device__ Producer(const Ctx &cc, uint32_t id) : c(cc), s(0), pid(id), ok(true), l2_only(id == (uint32_t)kProducerWarps) {}
+  __device__ __forceinline__ bool mine() const { return l2_only || s % (uint32_t)kProducerWarps == pid; }
+  // prefetcher: stay at most l2_window stages ahead of the ring (producer 0's count)
+  __device__ __forceinline__ bool throttle() {
+    const uint32_t win = c.p->l2_window;
+    if (s > *c.progress + win && !*c.abort_flag) {
+      const uint64_t t0 = now_ns();
+      for (uint32_t it = 1; s > *c.progress + win && !*c.abort_flag; ++it) {
+        __nanosleep(100);
+        if ((it & 63u) == 0u && now_ns() - t0 > c.p->wait_ns) raise_timeout(c);
+      }
+    }
+    if (*c.abort_flag) { ok = false; return false; }
+    return true;
+  }
   // Wait until the slot of stage s is free.  Successive fills of a slot are issued by
   // different warps, so the release counter (not the parity alone) says which fill
   // was consumed; the mbarrier wait that follows orders the consumers' reads before
@@ -259,8 +282,14 @@ struct Producer {
         const int kw = min(kChunk, ph.K - kc * kChunk);
         for (int ww = 0; ww < nw; ++ww, ++s) {
           if (!mine()) continue;
+          if (l2_only) {
+            if (!throttle()) return;
+            if (w == ww) l2_prefetch(row + (size_t)kc * kChunk, (uint32_t)kw * 2u);
+            continue;
+          }
           uint32_t slot;
           if (!acquire(slot)) return;
+          if (pid == 0 && lane == 0) *c.progress = s;
           const uint32_t bar = smem_u32(&c.full[slot]);
           // the copies may complete bytes before the expect_tx lands: the phase cannot
           // end before its one arrival (the expect_tx itself)
@@ -282,10 +311,18 @@ struct Producer {
       if (chunk == a.nch - 1) continue;   // the chunk with the current position: plain loads
       const int kvh = stream / qgroups;
       if (!mine()) { ++s; continue; }
-      uint32_t slot;
-      if (!acquire(slot)) return;
       const size_t off = ((((size_t)layer * dm.max_slots + p.slot) * dm.Hkv + kvh) * dm.max_seq +
                           (size_t)chunk * a.CH) * dm.dh;
+      if (l2_only) {
+        if (!throttle()) return;
+        if (lane == 0) l2_prefetch(p.Kc + off, kStageBytes / 2);
+        if (lane == 1) l2_prefetch(p.Vc + off, kStageBytes / 2);
+        ++s;
+        continue;
+      }
+      uint32_t slot;
+      if (!acquire(slot)) return;
+      if (pid == 0 && lane == 0) *c.progress = s;
       const uint32_t bar = smem_u32(&c.full[slot]);
       const uint32_t dst = smem_u32(c.ring + (size_t)slot * kStageBytes);
       if (lane == 0) mbar_expect_tx(bar, (uint32_t)kStageBytes);
@@ -699,6 +736,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) k_step_b1(const __grid_const
   __shared__ __align__(8) uint64_t s_full[kMaxStages], s_empty[kMaxStages];
   __shared__ uint32_t s_released[kMaxStages];
   __shared__ int s_abort;
+  __shared__ uint32_t s_progress;
   __shared__ __align__(16) float s_x_own[kMaxOwnRows];
   __shared__ float2 s_rope[64];
   const int tid = threadIdx.x, warp = tid >> 5;
@@ -709,11 +747,13 @@ __global__ void __launch_bounds__(kFusedThreads, 1) k_step_b1(const __grid_const
   c.full = s_full; c.empty = s_empty;
   c.released = s_released;
   c.abort_flag = &s_abort;
+  c.progress = &s_progress;
   c.x_own = s_x_own;
   c.rope_row = s_rope;
   c.cta = blockIdx.x; c.ncta = gridDim.x;
   if (tid == 0) {
     s_abort = 0;
+    s_progress = 0;
     for (int i = 0; i < p.n_stages; ++i) {
       s_released[i] = 0;
       mbar_init(smem_u32(&s_full[i]), 1);
@@ -738,6 +778,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) k_step_b1(const __grid_const
   if (warp >= 8) {
     // ------------------------------------------------------------ producers
     Producer pr(c, (uint32_t)(warp - 8));
+    if (pr.l2_only && p.l2_window == 0) return;   // look-ahead switched off
     for (int l = 0; l < L && pr.ok; ++l) {
       if (lo <= l && l < hi) continue;
       pr.gemv_phase(make_phase(p, PH_QKV, l, c.cta, c.ncta));
@@ -747,7 +788,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) k_step_b1(const __grid_const
       pr.gemv_phase(make_phase(p, PH_DOWN, l, c.cta, c.ncta));
     }
     if (pr.ok && p.logits) pr.gemv_phase(make_phase(p, PH_HEAD, 0, c.cta, c.ncta));
-    if (!pr.ok && (tid & 31) == 0) {
+    if (!pr.ok && !pr.l2_only && (tid & 31) == 0) {
       // drain: wait (bounded) until every copy already issued has landed
       const uint32_t ns = (uint32_t)p.n_stages;
       const uint32_t first = pr.s > ns ? pr.s - ns : 0;
@@ -947,6 +988,16 @@ int fused_plan(const d3_config &c, int *grid, int *n_stages, int *act_floats, si
   if (!ok) return 0;
   *grid = pl.grid; *n_stages = pl.n_stages; *act_floats = pl.act_floats; *smem = pl.smem; *func = pl.func;
   return 1;
+}
+
+uint32_t fused_l2_window() {
+  // 24 stages of 16 KB per CTA: ~58 MB over 148 CTAs, about 9 us of HBM time, inside the 126 MB L2
+  uint32_t w = 24;
+  if (const char *env = getenv("D3_FUSED_L2_WINDOW")) {
+    const int v = atoi(env);
+    if (v == 0 || (v >= 4 && v <= 256)) w = (uint32_t)v;   // below 4 the prefetcher could not finish
+  }
+  return w;
 }
 
 int launch_fused_step(void *func, int grid, size_t smem, FusedParams &fp, cudaStream_t st) {

@@ -100,6 +100,7 @@ struct FusedParams {
   float *x, *qkv, *u, *part, *attn_out;
   float *logits;
   int32_t n_stages, act_floats;
+  uint32_t l2_window;           // ring stages the L2 prefetcher may run ahead (0 = off)
   unsigned long long wait_ns;   // bound of every device-side wait
 };
 
@@ -131,5 +132,6 @@ int init_kernel_attributes();
 // fused batch-1 step: returns 1 and the launch plan when the kernel serves `c` on this device
 int fused_plan(const d3_config &c, int *grid, int *n_stages, int *act_floats, size_t *smem, void **func);
 int launch_fused_step(void *func, int grid, size_t smem, FusedParams &fp, cudaStream_t st);
+uint32_t fused_l2_window();   // look-ahead of the L2 prefetcher in ring stages (D3_FUSED_L2_WINDOW overrides)
 
 }  // namespace d3
