@@ -46,6 +46,8 @@ constexpr int kStageBytes = 16384;
 constexpr int kChunk = 2048;          // weight elements of one row segment
 constexpr int kMaxStages = 14;
 constexpr int kMaxGQ = 4;
+constexpr int kAttParts = 4;          // CTAs that share one attention stream, at most
+constexpr int kMaxHeads = 128;        // query heads the merge scratch is sized for
 constexpr int kMaxOwnRows = 1024;     // residual-stream rows one CTA may own (d / #CTAs, rounded up)
 
 enum PhaseKind { PH_QKV = 0, PH_OPROJ, PH_GATEUP, PH_DOWN, PH_HEAD };
@@ -201,29 +203,25 @@ __device__ __forceinline__ const bf16 *group_row(const Phase &ph, const Dims &dm
 // Streams: (kv head, group of GQ query heads).  A stream's positions 0..pos are
 // cut into chunks of CH positions (8 KB of K); the last chunk holds the current
 // position and is read with plain loads after the grid barrier, the others go
-// through the ring.  Units u = stream * nch + chunk are dealt to CTAs in
-// contiguous ranges.
-struct AttSplit {
-  int CH, nch, streams, units, u0, u1, gq;
+// through the ring.  Every stream is served by P CTAs (a fixed number, so that
+// the merge after the barrier is a fully unrolled, single-round-trip load): part
+// k of stream s takes the chunks [nch*k/P, nch*(k+1)/P) and belongs to CTA
+// (s*P + k) mod #CTAs.  A part may be empty; it still writes an (empty) partial.
+struct AttPlan {
+  int CH, nch, streams, P, parts, gq;
 };
 
-__device__ __forceinline__ AttSplit make_att(const FusedParams &p, int gq, int cta, int ncta) {
-  AttSplit a;
+__device__ __forceinline__ AttPlan make_att(const FusedParams &p, int gq, int ncta) {
+  AttPlan a;
   a.gq = gq;
   a.CH = (kStageBytes / 2) / (p.dm.dh * 2);
   a.nch = p.pos / a.CH + 1;
   a.streams = p.dm.Hkv * ((p.dm.Hq / p.dm.Hkv) / gq);
-  a.units = a.streams * a.nch;
-  split_range(a.units, cta, ncta, a.u0, a.u1);
+  a.P = ncta / a.streams;
+  if (a.P > kAttParts) a.P = kAttParts;
+  if (a.P < 1) a.P = 1;
+  a.parts = a.streams * a.P;
   return a;
-}
-
-__device__ __forceinline__ int cta_of_unit(int u, int units, int ncta) {
-  int c = (int)(((long long)u * ncta) / units);
-  if (c >= ncta) c = ncta - 1;
-  while (c + 1 < ncta && (int)(((long long)units * (c + 1)) / ncta) <= u) ++c;
-  while (c > 0 && (int)(((long long)units * c) / ncta) > u) --c;
-  return c;
 }
 
 // ---- producers (all 32 lanes of each producer warp run this) ----------------------
@@ -301,34 +299,37 @@ struct Producer {
       }
     }
   }
-  __device__ void att_phase(const AttSplit &a, int layer) {
+  __device__ void att_phase(const AttPlan &a, int layer) {
     const FusedParams &p = *c.p;
     const Dims &dm = p.dm;
     const int lane = threadIdx.x & 31;
     const int G = dm.Hq / dm.Hkv, qgroups = G / a.gq;
-    for (int u = a.u0; u < a.u1 && ok; ++u) {
-      const int stream = u / a.nch, chunk = u % a.nch;
-      if (chunk == a.nch - 1) continue;   // the chunk with the current position: plain loads
+    for (int part = c.cta; part < a.parts && ok; part += c.ncta) {
+      const int stream = part / a.P, k = part % a.P;
       const int kvh = stream / qgroups;
-      if (!mine()) { ++s; continue; }
-      const size_t off = ((((size_t)layer * dm.max_slots + p.slot) * dm.Hkv + kvh) * dm.max_seq +
-                          (size_t)chunk * a.CH) * dm.dh;
-      if (l2_only) {
-        if (!throttle()) return;
-        if (lane == 0) l2_prefetch(p.Kc + off, kStageBytes / 2);
-        if (lane == 1) l2_prefetch(p.Vc + off, kStageBytes / 2);
+      const int ch0 = a.nch * k / a.P, ch1 = a.nch * (k + 1) / a.P;
+      for (int chunk = ch0; chunk < ch1; ++chunk) {
+        if (chunk == a.nch - 1) continue;   // the chunk with the current position: plain loads
+        if (!mine()) { ++s; continue; }
+        const size_t off = ((((size_t)layer * dm.max_slots + p.slot) * dm.Hkv + kvh) * dm.max_seq +
+                            (size_t)chunk * a.CH) * dm.dh;
+        if (l2_only) {
+          if (!throttle()) return;
+          if (lane == 0) l2_prefetch(p.Kc + off, kStageBytes / 2);
+          if (lane == 1) l2_prefetch(p.Vc + off, kStageBytes / 2);
+          ++s;
+          continue;
+        }
+        uint32_t slot;
+        if (!acquire(slot)) return;
+        if (pid == 0 && lane == 0) *c.progress = s;
+        const uint32_t bar = smem_u32(&c.full[slot]);
+        const uint32_t dst = smem_u32(c.ring + (size_t)slot * kStageBytes);
+        if (lane == 0) mbar_expect_tx(bar, (uint32_t)kStageBytes);
+        if (lane == 0) bulk_g2s(dst, p.Kc + off, kStageBytes / 2, bar);
+        if (lane == 1) bulk_g2s(dst + kStageBytes / 2, p.Vc + off, kStageBytes / 2, bar);
         ++s;
-        continue;
       }
-      uint32_t slot;
-      if (!acquire(slot)) return;
-      if (pid == 0 && lane == 0) *c.progress = s;
-      const uint32_t bar = smem_u32(&c.full[slot]);
-      const uint32_t dst = smem_u32(c.ring + (size_t)slot * kStageBytes);
-      if (lane == 0) mbar_expect_tx(bar, (uint32_t)kStageBytes);
-      if (lane == 0) bulk_g2s(dst, p.Kc + off, kStageBytes / 2, bar);
-      if (lane == 1) bulk_g2s(dst + kStageBytes / 2, p.Vc + off, kStageBytes / 2, bar);
-      ++s;
     }
   }
 };
@@ -542,41 +543,46 @@ struct Consumer {
     }
   }
 
-  // Attention of this CTA's units.  Each stream segment yields one partial
-  // (max, sum, o) in part[(stream * ncta + cta)][gq][dh + 2]; the CTA whose
-  // arrival completes a stream merges the stream's partials into attn_out.
+  // Attention of this CTA's parts.  Each part yields one partial (max, sum,
+  // unnormalised o) in part[stream * P + k][gq][dh + 2]; the partials are merged
+  // by merge_load_attn after the grid barrier.
   template <int DH, int GQ>
-  __device__ void att_phase(const AttSplit &a, int layer, unsigned ordinal) {
+  __device__ void att_phase(const AttPlan &a, int layer) {
     const FusedParams &p = *c.p;
     const Dims &dm = p.dm;
     constexpr int EPL = DH / 8;
-    __shared__ int s_nseg, s_last;
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, part = lane & 7;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, part8 = lane & 7;
     const int worker = warp * 4 + (lane >> 3);
     // the 8 lanes of a worker run the position loop in lockstep; other workers of
     // the warp may run fewer iterations, so in-loop shuffles name only the worker
     const unsigned wmask = 0xffu << (lane & 24);
     const int G = dm.Hq / dm.Hkv, qgroups = G / GQ;
     const float scale = rsqrtf((float)DH);
-    int u = a.u0;
     uint32_t ring_k = 0;   // ring stages of this phase seen so far (every warp counts them all)
-    while (u < a.u1) {
-      const int stream = u / a.nch;
+    for (int part = c.cta; part < a.parts; part += c.ncta) {
+      const int stream = part / a.P, kpart = part % a.P;
       const int kvh = stream / qgroups, qg = stream % qgroups;
       const int h0 = kvh * G + qg * GQ;
-      const int u_end = min(a.u1, (stream + 1) * a.nch);
+      const int ch0 = a.nch * kpart / a.P, ch1 = a.nch * (kpart + 1) / a.P;
+      float *dst = p.part + (size_t)part * (GQ * (DH + 2));
+      if (ch0 == ch1) {   // nothing to do: an empty partial (weight 0 in the merge)
+        for (int i = tid; i < GQ * (DH + 2); i += kConsumers) {
+          const int e = i % (DH + 2);
+          dst[i] = (e == DH) ? -INFINITY : 0.f;
+        }
+        continue;
+      }
       float q[GQ][EPL], mx[GQ], sum[GQ], o[GQ][EPL];
 #pragma unroll
       for (int g = 0; g < GQ; ++g) {
         mx[g] = -INFINITY; sum[g] = 0.f;
 #pragma unroll
         for (int e = 0; e < EPL; ++e) {
-          q[g][e] = __ldcg(p.qkv + (h0 + g) * DH + part * EPL + e) * scale;
+          q[g][e] = __ldcg(p.qkv + (h0 + g) * DH + part8 * EPL + e) * scale;
           o[g][e] = 0.f;
         }
       }
-      for (; u < u_end; ++u) {
-        const int chunk = u % a.nch;
+      for (int chunk = ch0; chunk < ch1; ++chunk) {
         const bool tail = chunk == a.nch - 1;
         // a ring stage belongs to one warp (its 4 workers walk the CH positions); the
         // tail chunk is read from global memory by all 32 workers
@@ -595,8 +601,8 @@ struct Consumer {
         for (int i = i0; i < cnt; i += istep) {
           float kf[EPL], vf[EPL];
           if (tail) {
-            const bf16 *kp = p.Kc + goff + (size_t)i * DH + part * EPL;
-            const bf16 *vp = p.Vc + goff + (size_t)i * DH + part * EPL;
+            const bf16 *kp = p.Kc + goff + (size_t)i * DH + part8 * EPL;
+            const bf16 *vp = p.Vc + goff + (size_t)i * DH + part8 * EPL;
 #pragma unroll
             for (int e = 0; e < EPL; e += 4) {
               const uint2 kw = __ldcg(reinterpret_cast<const uint2 *>(kp + e));
@@ -605,7 +611,7 @@ struct Consumer {
               vf[e] = bfl(vw.x); vf[e + 1] = bfh(vw.x); vf[e + 2] = bfl(vw.y); vf[e + 3] = bfh(vw.y);
             }
           } else {
-            const unsigned char *ks = c.ring + (size_t)slot * kStageBytes + ((size_t)i * DH + part * EPL) * 2;
+            const unsigned char *ks = c.ring + (size_t)slot * kStageBytes + ((size_t)i * DH + part8 * EPL) * 2;
             const unsigned char *vs = ks + kStageBytes / 2;
 #pragma unroll
             for (int e = 0; e < EPL; e += 4) {
@@ -655,20 +661,16 @@ struct Consumer {
       // the activation buffer is free during attention: it holds the merge scratch
       float *s_o = c.act;                       // [8][GQ][DH]
       float *s_ml = c.act + 8 * GQ * DH;        // [8][GQ][2]
-      int *s_list = reinterpret_cast<int *>(c.act + 8 * GQ * (DH + 2));   // CTAs holding a partial
-      float *s_pm = c.act + 8 * GQ * (DH + 2) + kFusedMaxCtas;            // [seg][kMaxGQ] max
-      float *s_pl = s_pm + kFusedMaxCtas * kMaxGQ;                        // [seg][kMaxGQ] sum
       consumer_sync();
       if (lane < 8) {
 #pragma unroll
         for (int g = 0; g < GQ; ++g) {
 #pragma unroll
-          for (int e = 0; e < EPL; ++e) s_o[(warp * GQ + g) * DH + part * EPL + e] = o[g][e];
+          for (int e = 0; e < EPL; ++e) s_o[(warp * GQ + g) * DH + part8 * EPL + e] = o[g][e];
           if (lane == 0) { s_ml[(warp * GQ + g) * 2] = mx[g]; s_ml[(warp * GQ + g) * 2 + 1] = sum[g]; }
         }
       }
       consumer_sync();
-      float *dst = p.part + ((size_t)stream * c.ncta + c.cta) * (GQ * (DH + 2));
       for (int i = tid; i < GQ * DH; i += kConsumers) {
         const int g = i / DH, e = i % DH;
         float M = -INFINITY;
@@ -686,47 +688,68 @@ struct Consumer {
         if (e == 0) { dst[g * (DH + 2) + DH] = M; dst[g * (DH + 2) + DH + 1] = Ls; }
       }
       consumer_sync();
-      // Publish the partial.  The CTA whose arrival completes the stream merges all
-      // of the stream's partials into attn_out; the others go on to the barrier.
-      if (tid == 0) {
-        const int c0 = cta_of_unit(stream * a.nch, a.units, c.ncta);
-        const int c1 = cta_of_unit((stream + 1) * a.nch - 1, a.units, c.ncta);
-        int nseg = 0;
-        for (int cc = c0; cc <= c1; ++cc)   // a CTA with an empty range wrote nothing
-          if ((long long)a.units * cc / c.ncta != (long long)a.units * (cc + 1) / c.ncta) s_list[nseg++] = cc;
-        __threadfence();
-        const unsigned old = atomicAdd(p.stream_count + stream, 1u);
-        s_nseg = nseg;
-        s_last = (old + 1u == (unsigned)nseg * ordinal) ? 1 : 0;
-      }
-      consumer_sync();
-      if (s_last) {
-        __threadfence();
-        const int nseg = s_nseg;
-        for (int i = tid; i < nseg * GQ; i += kConsumers) {
-          const int sg = i / GQ, g = i % GQ;
-          const float *src = p.part + ((size_t)stream * c.ncta + s_list[sg]) * (GQ * (DH + 2)) + g * (DH + 2);
-          s_pm[sg * kMaxGQ + g] = __ldcg(src + DH);
-          s_pl[sg * kMaxGQ + g] = __ldcg(src + DH + 1);
-        }
-        consumer_sync();
-        for (int i = tid; i < GQ * DH; i += kConsumers) {
-          const int g = i / DH, e = i % DH;
-          float M = -INFINITY;
-          for (int sg = 0; sg < nseg; ++sg) M = fmaxf(M, s_pm[sg * kMaxGQ + g]);
-          float Ls = 0.f, O = 0.f;
-#pragma unroll 4
-          for (int sg = 0; sg < nseg; ++sg) {
-            const float cf = __expf(s_pm[sg * kMaxGQ + g] - M);
-            Ls += s_pl[sg * kMaxGQ + g] * cf;
-            O += __ldcg(p.part + ((size_t)stream * c.ncta + s_list[sg]) * (GQ * (DH + 2)) + g * (DH + 2) + e) * cf;
-          }
-          p.attn_out[(h0 + g) * DH + e] = O / Ls;
-        }
-      }
-      consumer_sync();
     }
     s += ring_k;
+  }
+
+  // act := attention output of all heads, merged from the P partials of every stream
+  // (after the grid barrier).  All loads are issued before the first is used.
+  template <int DH, int GQ>
+  __device__ void merge_load_attn(const AttPlan &a, float *s_pm, float *s_pl) {
+    const FusedParams &p = *c.p;
+    const Dims &dm = p.dm;
+    const int tid = threadIdx.x;
+    const int G = dm.Hq / dm.Hkv, qgroups = G / GQ;
+    const int n_out = dm.Hq * DH, P = a.P;
+    // (max, sum) of every (head, part): entry h * kAttParts + k
+    for (int idx = tid; idx < dm.Hq * P; idx += kConsumers) {
+      const int h = idx / P, k = idx % P;
+      const int kvh = h / G, qg = (h % G) / GQ, g = (h % G) % GQ;
+      const float *src = p.part + (size_t)((kvh * qgroups + qg) * P + k) * (GQ * (DH + 2)) + g * (DH + 2);
+      s_pm[h * kAttParts + k] = __ldcg(src + DH);
+      s_pl[h * kAttParts + k] = __ldcg(src + DH + 1);
+    }
+    constexpr int kBatch = 16;
+    for (int j0 = 0; j0 * kConsumers < n_out; j0 += kBatch) {
+      float r[kBatch][kAttParts];
+#pragma unroll
+      for (int jj = 0; jj < kBatch; ++jj) {
+        const int i = (j0 + jj) * kConsumers + tid;
+#pragma unroll
+        for (int k = 0; k < kAttParts; ++k) {
+          r[jj][k] = 0.f;
+          if (i < n_out && k < P) {
+            const int h = i / DH, e = i % DH;
+            const int kvh = h / G, qg = (h % G) / GQ, g = (h % G) % GQ;
+            r[jj][k] = __ldcg(p.part + (size_t)((kvh * qgroups + qg) * P + k) * (GQ * (DH + 2)) +
+                              g * (DH + 2) + e);
+          }
+        }
+      }
+      if (j0 == 0) consumer_sync();   // the (max, sum) table is complete
+#pragma unroll
+      for (int jj = 0; jj < kBatch; ++jj) {
+        const int i = (j0 + jj) * kConsumers + tid;
+        if (i < n_out) {
+          const int h = i / DH;
+          float M = -INFINITY;
+#pragma unroll
+          for (int k = 0; k < kAttParts; ++k)
+            if (k < P) M = fmaxf(M, s_pm[h * kAttParts + k]);
+          float Ls = 0.f, O = 0.f;
+#pragma unroll
+          for (int k = 0; k < kAttParts; ++k) {
+            if (k < P) {
+              const float cf = __expf(s_pm[h * kAttParts + k] - M);   // exp(-inf) = 0 for an empty part
+              Ls += s_pl[h * kAttParts + k] * cf;
+              O += r[jj][k] * cf;
+            }
+          }
+          c.act[act_index(i)] = O / Ls;
+        }
+      }
+    }
+    consumer_sync();
   }
 };
 
@@ -737,6 +760,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) k_step_b1(const __grid_const
   __shared__ uint32_t s_released[kMaxStages];
   __shared__ int s_abort;
   __shared__ uint32_t s_progress;
+  __shared__ float s_pm[kMaxHeads * kAttParts], s_pl[kMaxHeads * kAttParts];
   __shared__ __align__(16) float s_x_own[kMaxOwnRows];
   __shared__ float2 s_rope[64];
   const int tid = threadIdx.x, warp = tid >> 5;
@@ -773,7 +797,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) k_step_b1(const __grid_const
   if (p.anchor == D3_ANCHOR_TAIL) { lo = n; hi = L; }
   else { if (n < p.start_id) n = p.start_id; lo = p.start_id; hi = p.start_id + (L - n); }
 
-  const AttSplit att = make_att(p, GQ, c.cta, c.ncta);
+  const AttPlan att = make_att(p, GQ, c.ncta);
 
   if (warp >= 8) {
     // ------------------------------------------------------------ producers
@@ -829,7 +853,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) k_step_b1(const __grid_const
     for (int i = tid; i < dm.dh / 2; i += kConsumers) s_rope[i] = p.rope[(size_t)p.pos * (dm.dh / 2) + i];
   }
   Consumer cs(c);
-  unsigned bidx = 0, ordinal = 0;
+  unsigned bidx = 0;
   // optional phase timer (thread 0 of every CTA): cycles spent up to each phase
   // boundary, summed in registers and written once at the end
   const bool timing = p.phase_cycles != nullptr && tid == 0;
@@ -863,11 +887,11 @@ __global__ void __launch_bounds__(kFusedThreads, 1) k_step_b1(const __grid_const
     tick(2);
     grid_barrier(c, ++bidx);
     tick(3);
-    cs.template att_phase<DH, GQ>(att, l, ++ordinal);
+    cs.template att_phase<DH, GQ>(att, l);
     tick(4);
     grid_barrier(c, ++bidx);
     tick(3);
-    load_act_plain(c, p.attn_out, dm.Hq * dm.dh);
+    cs.template merge_load_attn<DH, GQ>(att, s_pm, s_pl);
     tick(1);
     cs.gemv_phase(make_phase(p, PH_OPROJ, l, c.cta, c.ncta), l);
     tick(5);
@@ -946,9 +970,10 @@ static bool try_plan(FusedPlan &pl, const d3_config &c) {
   if (c.d_ffn > need) need = c.d_ffn;
   if (c.n_q_heads * c.head_dim > need) need = c.n_q_heads * c.head_dim;
   need = (need + kChunk - 1) / kChunk * kChunk;
-  const int att_need = 8 * kMaxGQ * (128 + 2) + kFusedMaxCtas * (1 + 2 * kMaxGQ);
+  const int att_need = 8 * kMaxGQ * (128 + 2);
+  if (c.n_q_heads > kMaxHeads) return false;
   if (need < att_need) need = (att_need + kChunk - 1) / kChunk * kChunk;
-  const int reserve = 8192;   // static shared memory of the kernel and slack
+  const int reserve = 12288;  // static shared memory of the kernel and slack
   int stages = (optin - reserve - need * 4) / kStageBytes;
   if (stages > kMaxStages) stages = kMaxStages;
   if (const char *env = getenv("D3_FUSED_STAGES")) {   // tuning knob: a shallower ring
@@ -991,8 +1016,9 @@ int fused_plan(const d3_config &c, int *grid, int *n_stages, int *act_floats, si
 }
 
 uint32_t fused_l2_window() {
-  // 24 stages of 16 KB per CTA: ~58 MB over 148 CTAs, about 9 us of HBM time, inside the 126 MB L2
-  uint32_t w = 24;
+  // 12 stages of 16 KB per CTA: ~29 MB over 148 CTAs, ~4.5 us of HBM time on top of the ring;
+  // measured: 8-16 help, 24 and more lose to L2 evictions before use
+  uint32_t w = 12;
   if (const char *env = getenv("D3_FUSED_L2_WINDOW")) {
     const int v = atoi(env);
     if (v == 0 || (v >= 4 && v <= 256)) w = (uint32_t)v;   // below 4 the prefetcher could not finish
