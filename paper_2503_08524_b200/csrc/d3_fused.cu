@@ -701,13 +701,21 @@ struct Consumer {
     const int tid = threadIdx.x;
     const int G = dm.Hq / dm.Hkv, qgroups = G / GQ;
     const int n_out = dm.Hq * DH, P = a.P;
-    // (max, sum) of every (head, part): entry h * kAttParts + k
-    for (int idx = tid; idx < dm.Hq * P; idx += kConsumers) {
-      const int h = idx / P, k = idx % P;
-      const int kvh = h / G, qg = (h % G) / GQ, g = (h % G) % GQ;
-      const float *src = p.part + (size_t)((kvh * qgroups + qg) * P + k) * (GQ * (DH + 2)) + g * (DH + 2);
-      s_pm[h * kAttParts + k] = __ldcg(src + DH);
-      s_pl[h * kAttParts + k] = __ldcg(src + DH + 1);
+    // (max, sum) of every (head, part), entry h * kAttParts + k: loaded into registers
+    // here, parked in shared memory only after the first batch of o loads is in flight
+    constexpr int kMl = (kMaxHeads * kAttParts + kConsumers - 1) / kConsumers;
+    float pm_r[kMl], pl_r[kMl];
+#pragma unroll
+    for (int q = 0; q < kMl; ++q) {
+      const int idx = q * kConsumers + tid;
+      pm_r[q] = 0.f; pl_r[q] = 0.f;
+      if (idx < dm.Hq * P) {
+        const int h = idx / P, k = idx % P;
+        const int kvh = h / G, qg = (h % G) / GQ, g = (h % G) % GQ;
+        const float *src = p.part + (size_t)((kvh * qgroups + qg) * P + k) * (GQ * (DH + 2)) + g * (DH + 2);
+        pm_r[q] = __ldcg(src + DH);
+        pl_r[q] = __ldcg(src + DH + 1);
+      }
     }
     constexpr int kBatch = 16;
     for (int j0 = 0; j0 * kConsumers < n_out; j0 += kBatch) {
@@ -726,7 +734,17 @@ struct Consumer {
           }
         }
       }
-      if (j0 == 0) consumer_sync();   // the (max, sum) table is complete
+      if (j0 == 0) {
+#pragma unroll
+        for (int q = 0; q < kMl; ++q) {
+          const int idx = q * kConsumers + tid;
+          if (idx < dm.Hq * P) {
+            s_pm[(idx / P) * kAttParts + idx % P] = pm_r[q];
+            s_pl[(idx / P) * kAttParts + idx % P] = pl_r[q];
+          }
+        }
+        consumer_sync();   // the (max, sum) table is complete
+      }
 #pragma unroll
       for (int jj = 0; jj < kBatch; ++jj) {
         const int i = (j0 + jj) * kConsumers + tid;
