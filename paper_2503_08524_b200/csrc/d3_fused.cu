@@ -699,7 +699,6 @@ struct Consumer {
     const FusedParams &p = *c.p;
     const Dims &dm = p.dm;
     const int tid = threadIdx.x;
-    const int G = dm.Hq / dm.Hkv, qgroups = G / GQ;
     const int n_out = dm.Hq * DH, P = a.P;
     // (max, sum) of every (head, part), entry h * kAttParts + k: loaded into registers
     // here, parked in shared memory only after the first batch of o loads is in flight
@@ -711,8 +710,8 @@ struct Consumer {
       pm_r[q] = 0.f; pl_r[q] = 0.f;
       if (idx < dm.Hq * P) {
         const int h = idx / P, k = idx % P;
-        const int kvh = h / G, qg = (h % G) / GQ, g = (h % G) % GQ;
-        const float *src = p.part + (size_t)((kvh * qgroups + qg) * P + k) * (GQ * (DH + 2)) + g * (DH + 2);
+        // heads are ordered [kv head][query group][g]: stream = h / GQ, g = h % GQ
+        const float *src = p.part + (size_t)((h / GQ) * P + k) * (GQ * (DH + 2)) + (h % GQ) * (DH + 2);
         pm_r[q] = __ldcg(src + DH);
         pl_r[q] = __ldcg(src + DH + 1);
       }
@@ -728,9 +727,7 @@ struct Consumer {
           r[jj][k] = 0.f;
           if (i < n_out && k < P) {
             const int h = i / DH, e = i % DH;
-            const int kvh = h / G, qg = (h % G) / GQ, g = (h % G) % GQ;
-            r[jj][k] = __ldcg(p.part + (size_t)((kvh * qgroups + qg) * P + k) * (GQ * (DH + 2)) +
-                              g * (DH + 2) + e);
+            r[jj][k] = __ldcg(p.part + (size_t)((h / GQ) * P + k) * (GQ * (DH + 2)) + (h % GQ) * (DH + 2) + e);
           }
         }
       }
