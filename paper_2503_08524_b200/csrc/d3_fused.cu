@@ -371,11 +371,23 @@ __device__ __forceinline__ void prefetch_gain(GainRegs &gr, const bf16 *gain, in
   }
 }
 
-// act := src (global fp32, length K), no normalisation
+// act := src (global fp32, length K), no normalisation.  Twelve 16-byte loads per
+// thread are in flight before the first is stored: one L2 round trip per 12 K floats.
 __device__ void load_act_plain(const Ctx &c, const float *src, int K) {
-#pragma unroll 4
-  for (int k = threadIdx.x * 4; k < K; k += kConsumers * 4)
-    *reinterpret_cast<float4 *>(c.act + act_index(k)) = ldcg4(src + k);
+  constexpr int kB = 12;
+  for (int k0 = 0; k0 < K; k0 += kB * kConsumers * 4) {
+    float4 v[kB];
+#pragma unroll
+    for (int q = 0; q < kB; ++q) {
+      const int k = k0 + q * (kConsumers * 4) + threadIdx.x * 4;
+      if (k < K) v[q] = ldcg4(src + k);
+    }
+#pragma unroll
+    for (int q = 0; q < kB; ++q) {
+      const int k = k0 + q * (kConsumers * 4) + threadIdx.x * 4;
+      if (k < K) *reinterpret_cast<float4 *>(c.act + act_index(k)) = v[q];
+    }
+  }
   consumer_sync();
 }
 
@@ -775,6 +787,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) k_step_b1(const __grid_const
   __shared__ uint32_t s_released[kMaxStages];
   __shared__ int s_abort;
   __shared__ uint32_t s_progress;
+  __shared__ long long s_tacc[kFusedPhases];
   __shared__ float s_pm[kMaxHeads * kAttParts], s_pl[kMaxHeads * kAttParts];
   __shared__ __align__(16) float s_x_own[kMaxOwnRows];
   __shared__ float2 s_rope[64];
@@ -814,7 +827,10 @@ __global__ void __launch_bounds__(kFusedThreads, 1) k_step_b1(const __grid_const
 
   const AttPlan att = make_att(p, GQ, c.ncta);
 
+  // Register budget by role (warps 8-11 and warps 0-3 / 4-7 are whole warpgroups): the
+  // copy-issuing warps need few registers, the consumers get what they give up.
   if (warp >= 8) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 40;");
     // ------------------------------------------------------------ producers
     Producer pr(c, (uint32_t)(warp - 8));
     if (pr.l2_only && p.l2_window == 0) return;   // look-ahead switched off
@@ -842,6 +858,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) k_step_b1(const __grid_const
   }
 
   // -------------------------------------------------------------- consumers
+  asm volatile("setmaxnreg.inc.sync.aligned.u32 232;");
   const int tok = p.tok_dev ? p.tok_dev[0] : p.tok;
   if (c.cta == 0 && tid == 0) {
     DevSched *s = p.sched;
@@ -870,18 +887,15 @@ __global__ void __launch_bounds__(kFusedThreads, 1) k_step_b1(const __grid_const
   Consumer cs(c);
   unsigned bidx = 0;
   // optional phase timer (thread 0 of every CTA): cycles spent up to each phase
-  // boundary, summed in registers and written once at the end
+  // boundary, summed in shared memory and written once at the end
   const bool timing = p.phase_cycles != nullptr && tid == 0;
   long long t_prev = clock64();
-  long long t_acc[kFusedPhases];
-#pragma unroll
-  for (int k = 0; k < kFusedPhases; ++k) t_acc[k] = 0;
+  if (timing)
+    for (int k = 0; k < kFusedPhases; ++k) s_tacc[k] = 0;
   auto tick = [&](int k) {
     if (timing) {
       const long long t = clock64();
-#pragma unroll
-      for (int q = 0; q < kFusedPhases; ++q)
-        if (q == k) t_acc[q] += t - t_prev;
+      s_tacc[k] += t - t_prev;
       t_prev = t;
     }
   };
@@ -956,9 +970,8 @@ __global__ void __launch_bounds__(kFusedThreads, 1) k_step_b1(const __grid_const
   }
   tick(8);
   if (timing) {
-    t_acc[9] = cs.ring_wait;
-#pragma unroll
-    for (int k = 0; k < kFusedPhases; ++k) p.phase_cycles[c.cta * kFusedPhases + k] += t_acc[k];
+    s_tacc[9] = cs.ring_wait;
+    for (int k = 0; k < kFusedPhases; ++k) p.phase_cycles[c.cta * kFusedPhases + k] += s_tacc[k];
   }
 }
 
