@@ -428,6 +428,7 @@ __device__ void load_flow_plain(const Ctx &c, const float *src, int K, uint32_t 
       }
       if (ok || !spin_again(c, t0, it)) break;
     }
+    if (k0 == 0) consumer_sync();   // every warp has left the phase that read the old act
 #pragma unroll
     for (int q = 0; q < kB; ++q) {
       const int k = k0 + q * (kConsumers * 4) + threadIdx.x * 4;
@@ -1129,6 +1130,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) k_step_b1(const __grid_const
     l = next;
   }
   // the residual stream before the final norm, for diagnostics: every CTA its own rows
+  consumer_sync();   // the last epilogues of the other warps have updated x_own
   for (int i = tid; i < (og1 - og0) * 4; i += kConsumers) p.x[og0 * 4 + i] = s_x_own[i];
   // COPY fill of a window that opens at block 0: zeros (nothing to wait for)
   if (p.kv_fill == D3_FILL_COPY && lo == 0) {
