@@ -32,8 +32,6 @@ Layout make_layout(const d3_config &c) {
   y.phase = off;    off = align_up(off + (size_t)kFusedMaxCtas * kFusedPhases * 8, 256);
   y.part_fused = off;
   off = align_up(off + (size_t)c.n_q_heads * kFusedMaxCtas * (c.head_dim + 2) * 4, 256);
-  y.flow_half = fused_flow_half_bytes(c);
-  y.flow = off;     off = align_up(off + 2 * y.flow_half, 256);
   y.total = off;
   return y;
 }
@@ -124,10 +122,10 @@ static const char *kProfNames[D3_PROF_KINDS] = {
     "schedule+embed", "norm+qkv", "rope+kv_append", "attention", "o_proj+resid", "norm+gate_up+swiglu",
     "down+resid", "kv_fill", "norm+lm_head", "fused_step",
     // phases inside the fused step kernel (mean over CTAs, nominal-clock ms)
-    "fused:prologue", "fused:x_and_u_loads", "fused:qkv", "fused:attn_merge_load", "fused:attention",
+    "fused:prologue", "fused:load_act", "fused:qkv", "fused:grid_barriers", "fused:attention",
     "fused:o_proj", "fused:gate_up", "fused:down", "fused:head+fill", "fused:ring_wait(warp0)",
-    // smallest and largest per-CTA time spent in the attention merge load
-    "fused:attn_merge_load_min", "fused:attn_merge_load_max"};
+    // smallest and largest per-CTA time spent in grid barriers
+    "fused:grid_barriers_min", "fused:grid_barriers_max"};
 
 // Scope that brackets one launch (or a launcher's pair of launches) with events.
 struct ProfScope {
@@ -287,7 +285,6 @@ static int32_t run_fused_step(d3_model *m, const StepArgs &a, float *logits_dev,
   fp.part = reinterpret_cast<float *>(m->scratch + m->lay.part_fused);
   fp.logits = logits_dev;
   fp.n_stages = m->fused_stages; fp.act_floats = m->fused_act;
-  fused_set_flow(fp, m->scratch + m->lay.flow, m->lay.flow_half, m->cfg);
   fp.l2_window = fused_l2_window();
   fp.wait_ns = 2000000000ull;
   int rc;

@@ -13,17 +13,10 @@
 // ring refills from L2 afterwards.  Each ring
 // stage is consumed by ONE of the warps 0-7 (stage s of a phase by warp s mod 8),
 // so the warps work on eight stages at a time and never synchronise inside a
-// projection.  The phases of a block (RMSNorm+QKV+RoPE+KV append | attention |
-// O-proj+residual | RMSNorm+gate/up+SwiGLU | down+residual) exchange only small
-// fp32 vectors between CTAs, through L2.  There is no grid barrier: every
-// exchanged float carries a 2-bit version tag in its two lowest mantissa bits
-// (a 2^-22 relative perturbation), buffers alternate between two copies, and a
-// reader simply reloads its elements until all of them show the tag of the
-// version it waits for.  A cross-CTA round trip costs 1-2 us on this part, a
-// counter barrier needs three of them in a row (publish, poll, load); data that
-// validates itself needs about one and a half.  Two copies suffice: whoever
-// writes version n+2 of a vector has consumed data that every reader of version
-// n produced after it finished reading.
+// projection.  Phases of a block (RMSNorm+QKV+RoPE+KV append | attention |
+// O-proj+residual | RMSNorm+gate/up+SwiGLU | down+residual) are separated by
+// grid barriers on a global counter; only the small fp32 activations cross them
+// (through L2, read with ld.global.cg).
 //
 // A ring stage is 16 KB: four weight-row segments of 2048 bf16 (a "row group" x
 // k-chunk), or 8 KB of K plus 8 KB of V for one KV head.  Row groups are issued
@@ -54,8 +47,7 @@ constexpr int kChunk = 2048;          // weight elements of one row segment
 constexpr int kMaxStages = 14;
 constexpr int kMaxGQ = 4;
 constexpr int kAttParts = 4;          // CTAs that share one attention stream, at most
-constexpr int kMaxHeads = 128;
-constexpr float kEmptyMax = -1e30f;   // running maximum of an attention partial without positions (finite: it carries a tag)        // query heads the merge scratch is sized for
+constexpr int kMaxHeads = 128;        // query heads the merge scratch is sized for
 constexpr int kMaxOwnRows = 1024;     // residual-stream rows one CTA may own (d / #CTAs, rounded up)
 
 enum PhaseKind { PH_QKV = 0, PH_OPROJ, PH_GATEUP, PH_DOWN, PH_HEAD };
@@ -93,6 +85,7 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void *src, uint32_t
       : "memory");
 }
 __device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+__device__ __forceinline__ float4 ldcg4(const float *p) { return __ldcg(reinterpret_cast<const float4 *>(p)); }
 __device__ __forceinline__ uint64_t now_ns() {
   uint64_t t;
   asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
@@ -134,48 +127,24 @@ __device__ __forceinline__ bool wait_bar(const Ctx &c, uint32_t bar, uint32_t pa
   return false;
 }
 
-// ---- self-validating exchange ---------------------------------------------------
-__device__ __forceinline__ void st_flow(float *p, float v, uint32_t tag) {
-  asm volatile("st.relaxed.gpu.global.u32 [%0], %1;" ::"l"(p), "r"((__float_as_uint(v) & ~3u) | tag) : "memory");
-}
-__device__ __forceinline__ uint4 ld_flow4(const float *p) {
-  uint4 v;
-  asm volatile("ld.relaxed.gpu.global.v4.u32 {%0,%1,%2,%3}, [%4];"
-               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
-               : "l"(p)
-               : "memory");
-  return v;
-}
-__device__ __forceinline__ uint32_t ld_flow1(const float *p) {
-  uint32_t v;
-  asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
-  return v;
-}
-__device__ __forceinline__ bool tag_ok(uint32_t v, uint32_t tag) { return (v & 3u) == tag; }
-__device__ __forceinline__ bool tag_ok4(uint4 v, uint32_t tag) {
-  return (((v.x ^ tag) | (v.y ^ tag) | (v.z ^ tag) | (v.w ^ tag)) & 3u) == 0u;
-}
-__device__ __forceinline__ float untag(uint32_t v) { return __uint_as_float(v & ~3u); }
-__device__ __forceinline__ float4 untag4(uint4 v) {
-  return make_float4(untag(v.x), untag(v.y), untag(v.z), untag(v.w));
-}
-// Wait (bounded) until one element shows the tag: a cheap poll of 4 bytes per thread
-// that precedes every full validated load, so that waiting CTAs do not flood L2.
-__device__ __forceinline__ void poll_one(const Ctx &c, const float *p, uint32_t tag);
-
-// one step of a bounded spin: false when the caller must stop (abort mode)
-__device__ __forceinline__ bool spin_again(const Ctx &c, uint64_t &t0, uint32_t &it) {
-  if (*c.abort_flag) return false;
-  if (it == 0) t0 = now_ns();
-  if ((++it & 15u) == 0u && now_ns() - t0 > c.p->wait_ns) { raise_timeout(c); return false; }
-  return true;
-}
-
-__device__ __forceinline__ void poll_one(const Ctx &c, const float *p, uint32_t tag) {
-  uint64_t t0 = 0;
-  uint32_t it = 0;
-  while (!tag_ok(ld_flow1(p), tag))
-    if (!spin_again(c, t0, it)) break;
+// Grid barrier number `idx` (1-based) among the consumer threads of all CTAs.
+// bar.sync orders the CTA's writes before thread 0; its release-add publishes them
+// at GPU scope; the acquire-load that sees the full count orders the other CTAs'
+// writes before everything after the second bar.sync.
+__device__ __forceinline__ void grid_barrier(const Ctx &c, unsigned idx) {
+  consumer_sync();
+  if (threadIdx.x == 0) {
+    asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(c.p->bar_counter) : "memory");
+    const unsigned target = idx * (unsigned)c.ncta;
+    const uint64_t t0 = now_ns();
+    for (uint32_t it = 1; !*c.abort_flag; ++it) {
+      unsigned v;
+      asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(c.p->bar_counter) : "memory");
+      if (v >= target) break;
+      if ((it & 15u) == 0u && now_ns() - t0 > c.p->wait_ns) raise_timeout(c);
+    }
+  }
+  consumer_sync();
 }
 
 // ---- the CTA's share of a phase ---------------------------------------------
@@ -402,95 +371,48 @@ __device__ __forceinline__ void prefetch_gain(GainRegs &gr, const bf16 *gain, in
   }
 }
 
-// act := version `tag` of the exchanged vector src (length K), no normalisation.
-// Eight 16-byte loads per thread are in flight per attempt.
-__device__ void load_flow_plain(const Ctx &c, const float *src, int K, uint32_t tag) {
-  constexpr int kB = 8;
-  {   // each thread watches one element, spread over the whole vector
-    const int nvec = K / 4;
-    poll_one(c, src + 4 * (int)(((long long)threadIdx.x * nvec) / kConsumers), tag);
-  }
+// act := src (global fp32, length K), no normalisation.  Twelve 16-byte loads per
+// thread are in flight before the first is stored: one L2 round trip per 12 K floats.
+__device__ void load_act_plain(const Ctx &c, const float *src, int K) {
+  constexpr int kB = 12;
   for (int k0 = 0; k0 < K; k0 += kB * kConsumers * 4) {
-    uint4 v[kB];
-    uint64_t t0 = 0;
-    uint32_t it = 0;
-    for (;;) {
-      bool ok = true;
-#pragma unroll
-      for (int q = 0; q < kB; ++q) {
-        const int k = k0 + q * (kConsumers * 4) + threadIdx.x * 4;
-        if (k < K) v[q] = ld_flow4(src + k);
-      }
-#pragma unroll
-      for (int q = 0; q < kB; ++q) {
-        const int k = k0 + q * (kConsumers * 4) + threadIdx.x * 4;
-        if (k < K) ok = ok && tag_ok4(v[q], tag);
-      }
-      if (ok || !spin_again(c, t0, it)) break;
-    }
-    if (k0 == 0) consumer_sync();   // every warp has left the phase that read the old act
+    float4 v[kB];
 #pragma unroll
     for (int q = 0; q < kB; ++q) {
       const int k = k0 + q * (kConsumers * 4) + threadIdx.x * 4;
-      if (k < K) *reinterpret_cast<float4 *>(c.act + act_index(k)) = untag4(v[q]);
+      if (k < K) v[q] = ldcg4(src + k);
+    }
+#pragma unroll
+    for (int q = 0; q < kB; ++q) {
+      const int k = k0 + q * (kConsumers * 4) + threadIdx.x * 4;
+      if (k < K) *reinterpret_cast<float4 *>(c.act + act_index(k)) = v[q];
     }
   }
   consumer_sync();
 }
 
-// act := RMSNorm(x) * gain, x = version `tag` of the exchanged vector src, or (src ==
-// nullptr) the bf16 embedding row `emb`.  Up to 4096 elements: the values wait in
-// registers for the scale.  Wider: sum of squares first, then a second pass (a
-// validated version does not change before it has been consumed by everybody).
-__device__ void load_flow_norm(const Ctx &c, const float *src, const bf16 *emb, int K, uint32_t tag,
-                               const GainRegs &gr, const bf16 *gain) {
+// act := RMSNorm(src) * gain.  Up to 4096 elements: one pass over L2, the values wait
+// in registers for the scale.  Wider: sum of squares first, then a second pass.
+__device__ void load_act_norm(const Ctx &c, const float *src, int K, const GainRegs &gr, const bf16 *gain) {
   const int tid = threadIdx.x;
   if (K <= GainRegs::kMaxIt * kConsumers * 4) {
     float4 v[GainRegs::kMaxIt];
-    if (src) {
-      poll_one(c, src + 4 * (int)(((long long)tid * (K / 4)) / kConsumers), tag);
-      uint4 raw[GainRegs::kMaxIt];
-      uint64_t t0 = 0;
-      uint32_t it = 0;
-      for (;;) {
-        bool ok = true;
-#pragma unroll
-        for (int q = 0; q < GainRegs::kMaxIt; ++q) {
-          const int k = q * (kConsumers * 4) + tid * 4;
-          if (k < K) raw[q] = ld_flow4(src + k);
-        }
-#pragma unroll
-        for (int q = 0; q < GainRegs::kMaxIt; ++q) {
-          const int k = q * (kConsumers * 4) + tid * 4;
-          if (k < K) ok = ok && tag_ok4(raw[q], tag);
-        }
-        if (ok || !spin_again(c, t0, it)) break;
-      }
-#pragma unroll
-      for (int q = 0; q < GainRegs::kMaxIt; ++q) v[q] = untag4(raw[q]);
-    } else {
-#pragma unroll
-      for (int q = 0; q < GainRegs::kMaxIt; ++q) {
-        const int k = q * (kConsumers * 4) + tid * 4;
-        if (k < K) {
-          const uint2 w = *reinterpret_cast<const uint2 *>(emb + k);
-          v[q] = make_float4(bfl(w.x), bfh(w.x), bfl(w.y), bfh(w.y));
-        }
-      }
-    }
     float ss = 0.f;
 #pragma unroll
-    for (int q = 0; q < GainRegs::kMaxIt; ++q) {
-      const int k = q * (kConsumers * 4) + tid * 4;
-      if (k < K) ss += v[q].x * v[q].x + v[q].y * v[q].y + v[q].z * v[q].z + v[q].w * v[q].w;
+    for (int it = 0; it < GainRegs::kMaxIt; ++it) {
+      const int k = it * (kConsumers * 4) + tid * 4;
+      if (k < K) {
+        v[it] = ldcg4(src + k);
+        ss += v[it].x * v[it].x + v[it].y * v[it].y + v[it].z * v[it].z + v[it].w * v[it].w;
+      }
     }
     const float scale = rsqrtf(block_sum(ss) / (float)K + c.p->eps);
 #pragma unroll
-    for (int q = 0; q < GainRegs::kMaxIt; ++q) {
-      const int k = q * (kConsumers * 4) + tid * 4;
+    for (int it = 0; it < GainRegs::kMaxIt; ++it) {
+      const int k = it * (kConsumers * 4) + tid * 4;
       if (k < K) {
-        float4 t = v[q];
-        const uint2 gw = gr.g[q];
+        float4 t = v[it];
+        const uint2 gw = gr.g[it];
         t.x *= scale * bfl(gw.x); t.y *= scale * bfh(gw.x);
         t.z *= scale * bfl(gw.y); t.w *= scale * bfh(gw.y);
         *reinterpret_cast<float4 *>(c.act + act_index(k)) = t;
@@ -499,30 +421,12 @@ __device__ void load_flow_norm(const Ctx &c, const float *src, const bf16 *emb, 
   } else {
     float ss = 0.f;
     for (int k = tid * 4; k < K; k += kConsumers * 4) {
-      float4 t;
-      if (src) {
-        uint4 raw;
-        uint64_t t0 = 0;
-        uint32_t it = 0;
-        for (;;) {
-          raw = ld_flow4(src + k);
-          if (tag_ok4(raw, tag) || !spin_again(c, t0, it)) break;
-        }
-        t = untag4(raw);
-      } else {
-        const uint2 w = *reinterpret_cast<const uint2 *>(emb + k);
-        t = make_float4(bfl(w.x), bfh(w.x), bfl(w.y), bfh(w.y));
-      }
+      const float4 t = ldcg4(src + k);
       ss += t.x * t.x + t.y * t.y + t.z * t.z + t.w * t.w;
     }
     const float scale = rsqrtf(block_sum(ss) / (float)K + c.p->eps);
     for (int k = tid * 4; k < K; k += kConsumers * 4) {
-      float4 t;
-      if (src) t = untag4(ld_flow4(src + k));
-      else {
-        const uint2 w = *reinterpret_cast<const uint2 *>(emb + k);
-        t = make_float4(bfl(w.x), bfh(w.x), bfl(w.y), bfh(w.y));
-      }
+      float4 t = ldcg4(src + k);
       const uint2 gw = *reinterpret_cast<const uint2 *>(gain + k);
       t.x *= scale * bfl(gw.x); t.y *= scale * bfh(gw.x);
       t.z *= scale * bfl(gw.y); t.w *= scale * bfh(gw.y);
@@ -536,9 +440,7 @@ struct Consumer {
   const Ctx &c;
   uint32_t s;     // ring stages of all finished phases (the same in every warp)
   long long ring_wait;   // cycles this thread spent waiting for ring stages (timing runs)
-  uint32_t nblk;         // executed blocks so far = version of q / kv / partials / u of the running block
-  int fill_src, fill_lo, fill_hi;   // COPY fill: blocks [fill_lo, fill_hi) get the K,V that block fill_src appends
-  __device__ Consumer(const Ctx &cc) : c(cc), s(0), ring_wait(0), nblk(0), fill_src(-1), fill_lo(0), fill_hi(0) {}
+  __device__ Consumer(const Ctx &cc) : c(cc), s(0), ring_wait(0) {}
 
   // Wait until stage number `sn` (counted over the whole step) has landed.
   // Stages of one slot are consumed by different warps, and a parity wait cannot
@@ -611,75 +513,45 @@ struct Consumer {
   __device__ void epilogue(const Phase &ph, const Dims &dm, int layer, int g, float y0, float y1, float y2,
                            float y3) {
     const FusedParams &p = *c.p;
-    const uint32_t tag = nblk & 3u, buf = nblk & 1u;
     if (ph.kind == PH_QKV) {
       const int per_head = dm.dh / 4, half = dm.dh / 2;
       const int rot_groups = (dm.Hq + dm.Hkv) * per_head;
-      const int nkv = dm.Hkv * dm.dh;
+      const size_t cbase = ((size_t)layer * dm.max_slots + p.slot) * dm.Hkv;
       if (g < rot_groups) {
         const int head = g / per_head, jj = (g % per_head) * 2;
         const float2 cs0 = c.rope_row[jj], cs1 = c.rope_row[jj + 1];
         const float a0 = y0 * cs0.x - y2 * cs0.y, b0 = y0 * cs0.y + y2 * cs0.x;
         const float a1 = y1 * cs1.x - y3 * cs1.y, b1 = y1 * cs1.y + y3 * cs1.x;
         if (head < dm.Hq) {
-          float *q = p.flow_q[buf] + head * dm.dh;
-          st_flow(q + jj, a0, tag); st_flow(q + jj + 1, a1, tag);
-          st_flow(q + jj + half, b0, tag); st_flow(q + jj + half + 1, b1, tag);
+          float *q = p.qkv + head * dm.dh;
+          q[jj] = a0; q[jj + 1] = a1; q[jj + half] = b0; q[jj + half + 1] = b1;
         } else {
-          const int hk = head - dm.Hq;
-          // this step's attention reads the new key from the exchange buffer (fp32)
-          float *kn = p.flow_kv[buf] + hk * dm.dh;
-          st_flow(kn + jj, a0, tag); st_flow(kn + jj + 1, a1, tag);
-          st_flow(kn + jj + half, b0, tag); st_flow(kn + jj + half + 1, b1, tag);
-          const bf16 k0 = __float2bfloat16_rn(a0), k1 = __float2bfloat16_rn(a1);
-          const bf16 k2 = __float2bfloat16_rn(b0), k3 = __float2bfloat16_rn(b1);
-          // the cache entry of this block, and of the dropped blocks it stands in for
-          // (written by the CTA that computed the values: no cross-CTA dependency)
-          int l2 = layer;
-          for (;;) {
-            bf16 *dst = p.Kc + ((((size_t)l2 * dm.max_slots + p.slot) * dm.Hkv + hk) * dm.max_seq + p.pos) * dm.dh;
-            dst[jj] = k0; dst[jj + 1] = k1; dst[jj + half] = k2; dst[jj + half + 1] = k3;
-            if (layer != fill_src) break;
-            l2 = (l2 == layer) ? fill_lo : l2 + 1;
-            if (l2 >= fill_hi) break;
-          }
+          bf16 *dst = p.Kc + ((cbase + (head - dm.Hq)) * dm.max_seq + p.pos) * dm.dh;
+          dst[jj] = __float2bfloat16_rn(a0); dst[jj + 1] = __float2bfloat16_rn(a1);
+          dst[jj + half] = __float2bfloat16_rn(b0); dst[jj + half + 1] = __float2bfloat16_rn(b1);
         }
       } else {
         const int r = (g - rot_groups) * 4, h = r / dm.dh, e = r % dm.dh;
-        float *vn = p.flow_kv[buf] + nkv + r;
-        st_flow(vn, y0, tag); st_flow(vn + 1, y1, tag); st_flow(vn + 2, y2, tag); st_flow(vn + 3, y3, tag);
-        const bf16 v0 = __float2bfloat16_rn(y0), v1 = __float2bfloat16_rn(y1);
-        const bf16 v2 = __float2bfloat16_rn(y2), v3 = __float2bfloat16_rn(y3);
-        int l2 = layer;
-        for (;;) {
-          bf16 *dst = p.Vc + ((((size_t)l2 * dm.max_slots + p.slot) * dm.Hkv + h) * dm.max_seq + p.pos) * dm.dh + e;
-          dst[0] = v0; dst[1] = v1; dst[2] = v2; dst[3] = v3;
-          if (layer != fill_src) break;
-          l2 = (l2 == layer) ? fill_lo : l2 + 1;
-          if (l2 >= fill_hi) break;
-        }
+        bf16 *dst = p.Vc + ((cbase + h) * dm.max_seq + p.pos) * dm.dh + e;
+        dst[0] = __float2bfloat16_rn(y0); dst[1] = __float2bfloat16_rn(y1);
+        dst[2] = __float2bfloat16_rn(y2); dst[3] = __float2bfloat16_rn(y3);
       }
     } else if (ph.kind == PH_GATEUP) {
-      float *u = p.flow_u[buf];
-      st_flow(u + 2 * g, y0 / (1.f + __expf(-y0)) * y2, tag);
-      st_flow(u + 2 * g + 1, y1 / (1.f + __expf(-y1)) * y3, tag);
+      p.u[2 * g] = y0 / (1.f + __expf(-y0)) * y2;
+      p.u[2 * g + 1] = y1 / (1.f + __expf(-y1)) * y3;
     } else if (ph.kind == PH_HEAD) {
       const int r = 4 * g;
       if (r < ph.R) p.logits[r] = y0;
       if (r + 1 < ph.R) p.logits[r + 1] = y1;
       if (r + 2 < ph.R) p.logits[r + 2] = y2;
       if (r + 3 < ph.R) p.logits[r + 3] = y3;
-    } else {   // O-proj / down: residual add on the rows this CTA owns (its own copy is
-               // current: no other CTA ever writes them), published for the others as
-               // version 2*nblk (after O-proj) or 2*nblk+1 (after down) of x
+    } else {   // O-proj / down: residual add on the rows this CTA owns (its own copy
+               // is current: no other CTA ever writes them), published for the others
       float4 *own = reinterpret_cast<float4 *>(c.x_own + 4 * (g - ph.g0));
       float4 v = *own;
       v.x += y0; v.y += y1; v.z += y2; v.w += y3;
       *own = v;
-      const uint32_t ver = 2u * nblk + (ph.kind == PH_DOWN ? 1u : 0u);
-      float *xo = p.flow_x[ver & 1u] + 4 * g;
-      st_flow(xo, v.x, ver & 3u); st_flow(xo + 1, v.y, ver & 3u);
-      st_flow(xo + 2, v.z, ver & 3u); st_flow(xo + 3, v.w, ver & 3u);
+      *reinterpret_cast<float4 *>(p.x + 4 * g) = v;
     }
   }
 
@@ -704,44 +576,22 @@ struct Consumer {
       const int kvh = stream / qgroups, qg = stream % qgroups;
       const int h0 = kvh * G + qg * GQ;
       const int ch0 = a.nch * kpart / a.P, ch1 = a.nch * (kpart + 1) / a.P;
-      const uint32_t tag = nblk & 3u, buf = nblk & 1u;
-      float *dst = p.flow_part[buf] + (size_t)part * (GQ * (DH + 2));
+      float *dst = p.part + (size_t)part * (GQ * (DH + 2));
       if (ch0 == ch1) {   // nothing to do: an empty partial (weight 0 in the merge)
         for (int i = tid; i < GQ * (DH + 2); i += kConsumers) {
           const int e = i % (DH + 2);
-          st_flow(dst + i, (e == DH) ? kEmptyMax : 0.f, tag);
+          dst[i] = (e == DH) ? -INFINITY : 0.f;
         }
         continue;
       }
       float q[GQ][EPL], mx[GQ], sum[GQ], o[GQ][EPL];
-      {   // the rotated queries of this block, as soon as every element shows the block's tag
-        uint4 raw[GQ][EPL / 4];
-        poll_one(c, p.flow_q[buf] + h0 * DH + part8 * EPL, tag);
-        uint64_t t0 = 0;
-        uint32_t it = 0;
-        for (;;) {
-          bool ok = true;
 #pragma unroll
-          for (int g = 0; g < GQ; ++g)
+      for (int g = 0; g < GQ; ++g) {
+        mx[g] = -INFINITY; sum[g] = 0.f;
 #pragma unroll
-            for (int e = 0; e < EPL / 4; ++e)
-              raw[g][e] = ld_flow4(p.flow_q[buf] + (h0 + g) * DH + part8 * EPL + e * 4);
-#pragma unroll
-          for (int g = 0; g < GQ; ++g)
-#pragma unroll
-            for (int e = 0; e < EPL / 4; ++e) ok = ok && tag_ok4(raw[g][e], tag);
-          if (ok || !spin_again(c, t0, it)) break;
-        }
-#pragma unroll
-        for (int g = 0; g < GQ; ++g) {
-          mx[g] = -INFINITY; sum[g] = 0.f;
-#pragma unroll
-          for (int e = 0; e < EPL / 4; ++e) {
-            const float4 f = untag4(raw[g][e]);
-            q[g][e * 4] = f.x * scale; q[g][e * 4 + 1] = f.y * scale;
-            q[g][e * 4 + 2] = f.z * scale; q[g][e * 4 + 3] = f.w * scale;
-            o[g][e * 4] = 0.f; o[g][e * 4 + 1] = 0.f; o[g][e * 4 + 2] = 0.f; o[g][e * 4 + 3] = 0.f;
-          }
+        for (int e = 0; e < EPL; ++e) {
+          q[g][e] = __ldcg(p.qkv + (h0 + g) * DH + part8 * EPL + e) * scale;
+          o[g][e] = 0.f;
         }
       }
       for (int chunk = ch0; chunk < ch1; ++chunk) {
@@ -762,35 +612,7 @@ struct Consumer {
         const size_t goff = ((((size_t)layer * dm.max_slots + p.slot) * dm.Hkv + kvh) * dm.max_seq + t0) * DH;
         for (int i = i0; i < cnt; i += istep) {
           float kf[EPL], vf[EPL];
-          if (tail && t0 + i == p.pos) {
-            // the token's own K,V: produced this step by other CTAs; read from the
-            // exchange buffer and rounded to the cache's bf16 like every other position
-            const float *kp = p.flow_kv[buf] + kvh * DH + part8 * EPL;
-            const float *vp = kp + dm.Hkv * DH;
-            uint4 kr[EPL / 4], vr[EPL / 4];
-            uint64_t ts = 0;
-            uint32_t it = 0;
-            for (;;) {
-              bool ok = true;
-#pragma unroll
-              for (int e = 0; e < EPL / 4; ++e) { kr[e] = ld_flow4(kp + e * 4); vr[e] = ld_flow4(vp + e * 4); }
-#pragma unroll
-              for (int e = 0; e < EPL / 4; ++e) ok = ok && tag_ok4(kr[e], tag) && tag_ok4(vr[e], tag);
-              if (ok || !spin_again(c, ts, it)) break;
-            }
-#pragma unroll
-            for (int e = 0; e < EPL / 4; ++e) {
-              const float4 kq = untag4(kr[e]), vq = untag4(vr[e]);
-              kf[e * 4] = __bfloat162float(__float2bfloat16_rn(kq.x));
-              kf[e * 4 + 1] = __bfloat162float(__float2bfloat16_rn(kq.y));
-              kf[e * 4 + 2] = __bfloat162float(__float2bfloat16_rn(kq.z));
-              kf[e * 4 + 3] = __bfloat162float(__float2bfloat16_rn(kq.w));
-              vf[e * 4] = __bfloat162float(__float2bfloat16_rn(vq.x));
-              vf[e * 4 + 1] = __bfloat162float(__float2bfloat16_rn(vq.y));
-              vf[e * 4 + 2] = __bfloat162float(__float2bfloat16_rn(vq.z));
-              vf[e * 4 + 3] = __bfloat162float(__float2bfloat16_rn(vq.w));
-            }
-          } else if (tail) {
+          if (tail) {
             const bf16 *kp = p.Kc + goff + (size_t)i * DH + part8 * EPL;
             const bf16 *vp = p.Vc + goff + (size_t)i * DH + part8 * EPL;
 #pragma unroll
@@ -874,8 +696,8 @@ struct Consumer {
           Ls += s_ml[(w * GQ + g) * 2 + 1] * cf;
           O += s_o[(w * GQ + g) * DH + e] * cf;
         }
-        st_flow(dst + g * (DH + 2) + e, O, tag);
-        if (e == 0) { st_flow(dst + g * (DH + 2) + DH, M, tag); st_flow(dst + g * (DH + 2) + DH + 1, Ls, tag); }
+        dst[g * (DH + 2) + e] = O;
+        if (e == 0) { dst[g * (DH + 2) + DH] = M; dst[g * (DH + 2) + DH + 1] = Ls; }
       }
       consumer_sync();
     }
@@ -883,75 +705,51 @@ struct Consumer {
   }
 
   // act := attention output of all heads, merged from the P partials of every stream
-  // as soon as they all show the block's tag.  All loads of an attempt are issued
-  // before the first is looked at.
+  // (after the grid barrier).  All loads are issued before the first is used.
   template <int DH, int GQ>
   __device__ void merge_load_attn(const AttPlan &a, float *s_pm, float *s_pl) {
     const FusedParams &p = *c.p;
     const Dims &dm = p.dm;
     const int tid = threadIdx.x;
     const int n_out = dm.Hq * DH, P = a.P;
-    const uint32_t tag = nblk & 3u;
-    const float *part = p.flow_part[nblk & 1u];
-    // (max, sum) of every (head, part), entry h * kAttParts + k
+    // (max, sum) of every (head, part), entry h * kAttParts + k: loaded into registers
+    // here, parked in shared memory only after the first batch of o loads is in flight
     constexpr int kMl = (kMaxHeads * kAttParts + kConsumers - 1) / kConsumers;
-    constexpr int kBatch = 8;
-    {   // each thread watches one element of one partial, spread over heads and parts
-      const int i = (int)(((long long)tid * n_out) / kConsumers), h = i / DH, e = i % DH, k = tid % P;
-      poll_one(c, part + (size_t)((h / GQ) * P + k) * (GQ * (DH + 2)) + (h % GQ) * (DH + 2) + e, tag);
+    float pm_r[kMl], pl_r[kMl];
+#pragma unroll
+    for (int q = 0; q < kMl; ++q) {
+      const int idx = q * kConsumers + tid;
+      pm_r[q] = 0.f; pl_r[q] = 0.f;
+      if (idx < dm.Hq * P) {
+        const int h = idx / P, k = idx % P;
+        // heads are ordered [kv head][query group][g]: stream = h / GQ, g = h % GQ
+        const float *src = p.part + (size_t)((h / GQ) * P + k) * (GQ * (DH + 2)) + (h % GQ) * (DH + 2);
+        pm_r[q] = __ldcg(src + DH);
+        pl_r[q] = __ldcg(src + DH + 1);
+      }
     }
+    constexpr int kBatch = 16;
     for (int j0 = 0; j0 * kConsumers < n_out; j0 += kBatch) {
-      uint32_t pm_r[kMl], pl_r[kMl];
-      uint32_t r[kBatch][kAttParts];
-      uint64_t t0 = 0;
-      uint32_t it = 0;
-      for (;;) {
-        bool ok = true;
-        if (j0 == 0) {
+      float r[kBatch][kAttParts];
 #pragma unroll
-          for (int q = 0; q < kMl; ++q) {
-            const int idx = q * kConsumers + tid;
-            if (idx < dm.Hq * P) {
-              const int h = idx / P, k = idx % P;
-              // heads are ordered [kv head][query group][g]: stream = h / GQ, g = h % GQ
-              const float *src = part + (size_t)((h / GQ) * P + k) * (GQ * (DH + 2)) + (h % GQ) * (DH + 2);
-              pm_r[q] = ld_flow1(src + DH);
-              pl_r[q] = ld_flow1(src + DH + 1);
-            }
+      for (int jj = 0; jj < kBatch; ++jj) {
+        const int i = (j0 + jj) * kConsumers + tid;
+#pragma unroll
+        for (int k = 0; k < kAttParts; ++k) {
+          r[jj][k] = 0.f;
+          if (i < n_out && k < P) {
+            const int h = i / DH, e = i % DH;
+            r[jj][k] = __ldcg(p.part + (size_t)((h / GQ) * P + k) * (GQ * (DH + 2)) + (h % GQ) * (DH + 2) + e);
           }
         }
-#pragma unroll
-        for (int jj = 0; jj < kBatch; ++jj) {
-          const int i = (j0 + jj) * kConsumers + tid;
-#pragma unroll
-          for (int k = 0; k < kAttParts; ++k) {
-            if (i < n_out && k < P) {
-              const int h = i / DH, e = i % DH;
-              r[jj][k] = ld_flow1(part + (size_t)((h / GQ) * P + k) * (GQ * (DH + 2)) + (h % GQ) * (DH + 2) + e);
-            }
-          }
-        }
-        if (j0 == 0) {
-#pragma unroll
-          for (int q = 0; q < kMl; ++q)
-            if (q * kConsumers + tid < dm.Hq * P) ok = ok && tag_ok(pm_r[q], tag) && tag_ok(pl_r[q], tag);
-        }
-#pragma unroll
-        for (int jj = 0; jj < kBatch; ++jj) {
-          const int i = (j0 + jj) * kConsumers + tid;
-#pragma unroll
-          for (int k = 0; k < kAttParts; ++k)
-            if (i < n_out && k < P) ok = ok && tag_ok(r[jj][k], tag);
-        }
-        if (ok || !spin_again(c, t0, it)) break;
       }
       if (j0 == 0) {
 #pragma unroll
         for (int q = 0; q < kMl; ++q) {
           const int idx = q * kConsumers + tid;
           if (idx < dm.Hq * P) {
-            s_pm[(idx / P) * kAttParts + idx % P] = untag(pm_r[q]);
-            s_pl[(idx / P) * kAttParts + idx % P] = untag(pl_r[q]);
+            s_pm[(idx / P) * kAttParts + idx % P] = pm_r[q];
+            s_pl[(idx / P) * kAttParts + idx % P] = pl_r[q];
           }
         }
         consumer_sync();   // the (max, sum) table is complete
@@ -961,7 +759,7 @@ struct Consumer {
         const int i = (j0 + jj) * kConsumers + tid;
         if (i < n_out) {
           const int h = i / DH;
-          float M = kEmptyMax;
+          float M = -INFINITY;
 #pragma unroll
           for (int k = 0; k < kAttParts; ++k)
             if (k < P) M = fmaxf(M, s_pm[h * kAttParts + k]);
@@ -969,9 +767,9 @@ struct Consumer {
 #pragma unroll
           for (int k = 0; k < kAttParts; ++k) {
             if (k < P) {
-              const float cf = __expf(s_pm[h * kAttParts + k] - M);   // 0 for an empty part
+              const float cf = __expf(s_pm[h * kAttParts + k] - M);   // exp(-inf) = 0 for an empty part
               Ls += s_pl[h * kAttParts + k] * cf;
-              O += untag(r[jj][k]) * cf;
+              O += r[jj][k] * cf;
             }
           }
           c.act[act_index(i)] = O / Ls;
@@ -1069,15 +867,25 @@ __global__ void __launch_bounds__(kFusedThreads, 1) k_step_b1(const __grid_const
     for (int l = 0; l < L; ++l) s->m[l] = (lo <= l && l < hi) ? 0 : 1;
     s->rows_layers = n; s->layers_touched = n;
   }
-  // embedding row -> residual stream: every CTA reads the row itself and keeps its own rows
+  // embedding row -> residual stream: CTA 0 publishes it, every CTA keeps its own rows
   const Dims &dm = p.dm;
   const bf16 *emb = p.embed + (size_t)tok * dm.d;
-  int og0, og1;
-  split_range(dm.d / 4, c.cta, c.ncta, og0, og1);
-  for (int i = tid; i < (og1 - og0) * 4; i += kConsumers) s_x_own[i] = __bfloat162float(emb[og0 * 4 + i]);
-  for (int i = tid; i < dm.dh / 2; i += kConsumers) s_rope[i] = p.rope[(size_t)p.pos * (dm.dh / 2) + i];
+  if (c.cta == 0) {
+    for (int k = tid * 8; k < dm.d; k += kConsumers * 8) {
+      const uint4 w = *reinterpret_cast<const uint4 *>(emb + k);
+      *reinterpret_cast<float4 *>(p.x + k) = make_float4(bfl(w.x), bfh(w.x), bfl(w.y), bfh(w.y));
+      *reinterpret_cast<float4 *>(p.x + k + 4) = make_float4(bfl(w.z), bfh(w.z), bfl(w.w), bfh(w.w));
+    }
+  }
+  {
+    int og0, og1;
+    split_range(dm.d / 4, c.cta, c.ncta, og0, og1);
+    for (int i = tid; i < (og1 - og0) * 4; i += kConsumers)
+      s_x_own[i] = __bfloat162float(emb[og0 * 4 + i]);
+    for (int i = tid; i < dm.dh / 2; i += kConsumers) s_rope[i] = p.rope[(size_t)p.pos * (dm.dh / 2) + i];
+  }
   Consumer cs(c);
-  if (p.kv_fill == D3_FILL_COPY && lo >= 1 && hi > lo) { cs.fill_src = lo - 1; cs.fill_lo = lo; cs.fill_hi = hi; }
+  unsigned bidx = 0;
   // optional phase timer (thread 0 of every CTA): cycles spent up to each phase
   // boundary, summed in shared memory and written once at the end
   const bool timing = p.phase_cycles != nullptr && tid == 0;
@@ -1097,58 +905,67 @@ __global__ void __launch_bounds__(kFusedThreads, 1) k_step_b1(const __grid_const
   GainRegs gr;
   const bf16 *gain = l < L ? p.layers[l].attn_norm : p.final_norm;
   prefetch_gain(gr, gain, dm.d);
-  consumer_sync();   // x_own and the rope row are in place
+  grid_barrier(c, ++bidx);
   tick(0);
-  // x entering a block: the embedding row (first block) or version 2*nblk-1 of x
   while (l < L) {
     int next = l + 1;   // dropped blocks: the hidden state passes through
     while (next < L && lo <= next && next < hi) ++next;
-    const uint32_t nb = cs.nblk;
-    load_flow_norm(c, nb ? p.flow_x[1] : nullptr, emb, dm.d, (2u * nb - 1u) & 3u, gr, gain);
+    load_act_norm(c, p.x, dm.d, gr, gain);
     tick(1);
     cs.gemv_phase(make_phase(p, PH_QKV, l, c.cta, c.ncta), l);
     tick(2);
+    grid_barrier(c, ++bidx);
+    tick(3);
     cs.template att_phase<DH, GQ>(att, l);
     tick(4);
-    cs.template merge_load_attn<DH, GQ>(att, s_pm, s_pl);
+    grid_barrier(c, ++bidx);
     tick(3);
+    cs.template merge_load_attn<DH, GQ>(att, s_pm, s_pl);
+    tick(1);
     cs.gemv_phase(make_phase(p, PH_OPROJ, l, c.cta, c.ncta), l);
     tick(5);
     gain = p.layers[l].mlp_norm;
     prefetch_gain(gr, gain, dm.d);
-    load_flow_norm(c, p.flow_x[0], nullptr, dm.d, (2u * nb) & 3u, gr, gain);
+    grid_barrier(c, ++bidx);
+    tick(3);
+    load_act_norm(c, p.x, dm.d, gr, gain);
     tick(1);
     cs.gemv_phase(make_phase(p, PH_GATEUP, l, c.cta, c.ncta), l);
     tick(6);
-    load_flow_plain(c, p.flow_u[nb & 1u], dm.f, nb & 3u);
+    grid_barrier(c, ++bidx);
+    tick(3);
+    load_act_plain(c, p.u, dm.f);
     tick(1);
     cs.gemv_phase(make_phase(p, PH_DOWN, l, c.cta, c.ncta), l);
     tick(7);
     gain = next < L ? p.layers[next].attn_norm : p.final_norm;
     prefetch_gain(gr, gain, dm.d);
-    cs.nblk = nb + 1u;
+    grid_barrier(c, ++bidx);
+    tick(3);
     l = next;
   }
-  // the residual stream before the final norm, for diagnostics: every CTA its own rows
-  consumer_sync();   // the last epilogues of the other warps have updated x_own
-  for (int i = tid; i < (og1 - og0) * 4; i += kConsumers) p.x[og0 * 4 + i] = s_x_own[i];
-  // COPY fill of a window that opens at block 0: zeros (nothing to wait for)
-  if (p.kv_fill == D3_FILL_COPY && lo == 0) {
+  // KV fill by copy for the dropped blocks: CTA j takes block lo + j, lo + j + ncta, ...
+  if (p.kv_fill == D3_FILL_COPY) {
     const int nkv = dm.Hkv * dm.dh;
     unsigned short *Ku = reinterpret_cast<unsigned short *>(p.Kc);
     unsigned short *Vu = reinterpret_cast<unsigned short *>(p.Vc);
-    for (int l2 = lo + c.cta; l2 < hi; l2 += c.ncta) {
+    for (int l = lo + c.cta; l < hi; l += c.ncta) {
       for (int i = tid; i < nkv; i += kConsumers) {
         const int h = i / dm.dh, e = i % dm.dh;
-        const size_t dst = ((((size_t)l2 * dm.max_slots + p.slot) * dm.Hkv + h) * dm.max_seq + p.pos) * dm.dh + e;
-        Ku[dst] = 0;
-        Vu[dst] = 0;
+        const size_t dst = ((((size_t)l * dm.max_slots + p.slot) * dm.Hkv + h) * dm.max_seq + p.pos) * dm.dh + e;
+        if (lo == 0) {
+          Ku[dst] = 0;
+          Vu[dst] = 0;
+        } else {
+          const size_t src = ((((size_t)(lo - 1) * dm.max_slots + p.slot) * dm.Hkv + h) * dm.max_seq + p.pos) * dm.dh + e;
+          Ku[dst] = __ldcg(Ku + src);   // written by another CTA earlier in this kernel
+          Vu[dst] = __ldcg(Vu + src);
+        }
       }
     }
   }
   if (p.logits) {
-    const uint32_t nb = cs.nblk;
-    load_flow_norm(c, nb ? p.flow_x[1] : nullptr, emb, dm.d, (2u * nb - 1u) & 3u, gr, gain);
+    load_act_norm(c, p.x, dm.d, gr, gain);
     cs.gemv_phase(make_phase(p, PH_HEAD, 0, c.cta, c.ncta), 0);
   }
   tick(8);
@@ -1226,28 +1043,6 @@ int fused_plan(const d3_config &c, int *grid, int *n_stages, int *act_floats, si
   return 1;
 }
 
-// one copy of the exchange buffers: x | q | k,v of the new token | u | attention partials
-size_t fused_flow_half_bytes(const d3_config &c) {
-  const size_t nq = (size_t)c.n_q_heads * c.head_dim, nkv = (size_t)c.n_kv_heads * c.head_dim;
-  const size_t floats = (size_t)c.d_model + nq + 2 * nkv + (size_t)c.d_ffn +
-                        (size_t)c.n_q_heads * kAttParts * (c.head_dim + 2);
-  return (floats * 4 + 255) / 256 * 256;
-}
-
-void fused_set_flow(FusedParams &fp, char *flow, size_t flow_half, const d3_config &c) {
-  const size_t nq = (size_t)c.n_q_heads * c.head_dim, nkv = (size_t)c.n_kv_heads * c.head_dim;
-  fp.flow_base = flow;
-  fp.flow_half_bytes = flow_half;
-  for (int b = 0; b < 2; ++b) {
-    float *f = reinterpret_cast<float *>(flow + (size_t)b * flow_half);
-    fp.flow_x[b] = f; f += c.d_model;
-    fp.flow_q[b] = f; f += nq;
-    fp.flow_kv[b] = f; f += 2 * nkv;
-    fp.flow_u[b] = f; f += c.d_ffn;
-    fp.flow_part[b] = f;
-  }
-}
-
 uint32_t fused_l2_window() {
   // 12 stages of 16 KB per CTA: ~29 MB over 148 CTAs, ~4.5 us of HBM time on top of the ring;
   // measured: 8-16 help, 24 and more lose to L2 evictions before use
@@ -1260,12 +1055,8 @@ uint32_t fused_l2_window() {
 }
 
 int launch_fused_step(void *func, int grid, size_t smem, FusedParams &fp, cudaStream_t st) {
-  // Exchange buffers start every step with tags no version will carry: the first copy
-  // sees versions with tags 0 and 2, the second with tags 1 and 3.
-  if (cudaMemsetAsync(fp.flow_base, 0x01, fp.flow_half_bytes, st) != cudaSuccess ||
-      cudaMemsetAsync(reinterpret_cast<char *>(fp.flow_base) + fp.flow_half_bytes, 0x02, fp.flow_half_bytes,
-                      st) != cudaSuccess)
-    return -1;
+  // grid-barrier counter and per-stream arrival counters start every step at zero
+  if (cudaMemsetAsync(fp.bar_counter, 0, kFusedSyncBytes, st) != cudaSuccess) return -1;
   void *args[] = {(void *)&fp};
   if (cudaLaunchCooperativeKernel(func, dim3(grid), dim3(kFusedThreads), args, smem, st) != cudaSuccess)
     return -1;

@@ -98,10 +98,6 @@ struct FusedParams {
   unsigned *stream_count;       // arrivals per attention stream
   long long *phase_cycles;      // nullable: [cta][kFusedPhases] cycles per phase
   float *x, *qkv, *u, *part, *attn_out;
-  // exchange buffers of the fused step, two copies each (see d3_fused.cu)
-  void *flow_base;
-  size_t flow_half_bytes;
-  float *flow_x[2], *flow_q[2], *flow_kv[2], *flow_u[2], *flow_part[2];
   float *logits;
   int32_t n_stages, act_floats;
   uint32_t l2_window;           // ring stages the L2 prefetcher may run ahead (0 = off)
@@ -110,7 +106,7 @@ struct FusedParams {
 
 // Byte offsets of the regions of the caller's scratch buffer.
 struct Layout {
-  size_t sched, rope, x, qkv, attn_out, part_o, part_ml, u, layer_tab, bar, phase, part_fused, flow, flow_half, total;
+  size_t sched, rope, x, qkv, attn_out, part_o, part_ml, u, layer_tab, bar, phase, part_fused, total;
   int max_splits;
 };
 
@@ -136,9 +132,6 @@ int init_kernel_attributes();
 // fused batch-1 step: returns 1 and the launch plan when the kernel serves `c` on this device
 int fused_plan(const d3_config &c, int *grid, int *n_stages, int *act_floats, size_t *smem, void **func);
 int launch_fused_step(void *func, int grid, size_t smem, FusedParams &fp, cudaStream_t st);
-uint32_t fused_l2_window();
-// point fp's exchange buffers into the scratch region at `flow` (two halves of flow_half bytes)
-void fused_set_flow(FusedParams &fp, char *flow, size_t flow_half, const d3_config &c);
-size_t fused_flow_half_bytes(const d3_config &c);   // look-ahead of the L2 prefetcher in ring stages (D3_FUSED_L2_WINDOW overrides)
+uint32_t fused_l2_window();   // look-ahead of the L2 prefetcher in ring stages (D3_FUSED_L2_WINDOW overrides)
 
 }  // namespace d3

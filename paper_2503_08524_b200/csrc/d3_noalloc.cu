@@ -122,7 +122,6 @@ extern "C" int32_t d3_decode_step_noalloc(const d3_config *cfg, const d3_weights
   fp.part = reinterpret_cast<float *>(scratch + lay.part_fused);
   fp.logits = logits_dev;
   fp.n_stages = stages; fp.act_floats = act;
-  fused_set_flow(fp, scratch + lay.flow, lay.flow_half, c1);
   fp.l2_window = fused_l2_window();
   fp.wait_ns = 2000000000ull;
   if (launch_fused_step(func, grid, smem, fp, st) != 1) return D3_ECUDA;
