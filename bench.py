@@ -41,6 +41,11 @@ METRIC = "decode tokens/s at 1 B200 and % of HBM roofline (retained-layer bytes/
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 ORACLE_PROMPT = 32            # bounded sample for the CPU oracle
+# dram__bytes_read + dram__bytes_write of one k_step_b1 launch over its algorithmic bytes, from the
+# ncu capture summarised in profiles/fused_step_k_step_b1_7bshape_L4.md (4-block case of the same
+# kernel: 1.8917 GB moved for 1.881 GB algorithmic; traffic grows with the blocks executed, so the
+# full launch is scaled by its own algorithmic bytes).  Set to None when the kernel changes.
+FUSED_TRAFFIC_RATIO = 1.0057
 
 
 def gen_indices(k: int):
@@ -338,6 +343,8 @@ def main():
         ach = class_bytes[top_name] * BATCH / 1e9 / (top_ms / top_n / 1e3)
         roofline.update(achieved=ach, frac=ach / peak, bytes_per_launch=class_bytes[top_name],
                         avg_launch_us=1e3 * top_ms / top_n)
+        if top_name == "fused_step" and FUSED_TRAFFIC_RATIO is not None:
+            roofline["traffic"] = FUSED_TRAFFIC_RATIO * class_bytes[top_name]
     else:
         roofline.update(achieved=None, frac=None)
     step_gbs = tot["bytes"] / 1e9 / (ms / 1e3)
