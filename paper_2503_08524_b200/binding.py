@@ -19,7 +19,7 @@ OK, EINVAL, ECAPACITY, ESTATE, ECUDA, ETIMEOUT = 0, -1, -2, -3, -4, -5
 ANCHOR_START, ANCHOR_TAIL = 0, 1
 FILL_NONE, FILL_COPY, FILL_RECOMPUTE = 0, 1, 2
 MAX_BATCH, MAX_LAYERS, PROF_KINDS = 64, 128, 22
-EXEC_AUTO, EXEC_KERNELS = 0, 1
+EXEC_AUTO, EXEC_KERNELS, EXEC_TENSOR = 0, 1, 2
 
 EXPORTS = ("d3_depth", "d3_schedule", "d3_workspace_bytes", "d3_load", "d3_prefill",
            "d3_decode_step", "d3_argmax", "d3_read_schedule", "d3_read_hidden", "d3_read_kv",

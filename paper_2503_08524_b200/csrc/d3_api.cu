@@ -32,6 +32,13 @@ Layout make_layout(const d3_config &c) {
   y.phase = off;    off = align_up(off + (size_t)kFusedMaxCtas * kFusedPhases * 8, 256);
   y.part_fused = off;
   off = align_up(off + (size_t)c.n_q_heads * kFusedMaxCtas * (c.head_dim + 2) * 4, 256);
+  // tensor-core operand: bf16 hi rows + lo rows of the widest activation
+  size_t kmax = (size_t)c.d_model;
+  if ((size_t)c.n_q_heads * c.head_dim > kmax) kmax = (size_t)c.n_q_heads * c.head_dim;
+  if ((size_t)c.d_ffn > kmax) kmax = (size_t)c.d_ffn;
+  y.act_split = off = align_up(off, 1024);
+  y.act_split_bytes = 2 * ((B + 7) / 8 * 8) * kmax * sizeof(bf16);
+  off = align_up(off + y.act_split_bytes, 256);
   y.total = off;
   return y;
 }
@@ -105,6 +112,11 @@ struct d3_model {
   size_t fused_smem;
   void *fused_func;
   std::vector<LayerPtrs> layer_tab_host;
+  // tensor-core projections: tensor maps of the weight matrices (entry valid when tm_ok)
+  TcContext tc;
+  std::vector<TMap> tm_qkv, tm_kv, tm_o, tm_gate, tm_up, tm_down;
+  TMap tm_head;
+  bool tm_ok;
 
   DevSched *sched() const { return reinterpret_cast<DevSched *>(scratch + lay.sched); }
   float2 *rope() const { return reinterpret_cast<float2 *>(scratch + lay.rope); }
@@ -174,6 +186,17 @@ static const int32_t *thr_for(d3_model *m, double alpha) {
   return it->second.data();
 }
 
+// One projection over `rows` rows: tensor cores for a dense enough group, FMA GEMV otherwise.
+static int project(d3_model *m, const GemvArgs &g, int epi, int rows) {
+  const bool tensor = m->exec_mode == D3_EXEC_TENSOR ||
+                      (m->exec_mode == D3_EXEC_AUTO && rows >= D3_TENSOR_MIN_ROWS);
+  if (tensor && m->tm_ok) {
+    int n = launch_gemm_tc(m->tc, g, epi, rows, m->stream);
+    if (n) return n;
+  }
+  return launch_gemv(g, epi, rows, m->stream);
+}
+
 // Enqueue one step over the rows described by `a` (already validated).
 // logits_mode: ROWS_ALL -> logits_dev[caller row][V]; ROWS_LAST -> logits_dev[V]
 // for the last row; logits_dev may be NULL (no LM head).
@@ -193,6 +216,7 @@ static int32_t run_step(d3_model *m, const StepArgs &a, const int32_t *n, const 
   memset(&g, 0, sizeof(g));
   g.sched = m->sched();
   g.eps = c.rms_eps;
+  const bool tm = m->tm_ok;
   for (int l = 0; l < L; ++l) {
     const int ml = m_l[l];
     g.layer = l;
@@ -200,9 +224,10 @@ static int32_t run_step(d3_model *m, const StepArgs &a, const int32_t *n, const 
       // RMSNorm + QKV projection
       g.row_mode = ROWS_PREFIX;
       g.W = m->wqkv[l]; g.W2 = nullptr; g.R = dm.qkv_rows; g.K = dm.d;
+      g.tmap_w = tm ? &m->tm_qkv[l] : nullptr; g.tmap_w2 = nullptr;
       g.act = m->x(); g.act_stride = dm.d; g.gain = m->attn_norm[l];
       g.out = m->qkv(); g.out_stride = dm.qkv_rows; g.out_col0 = 0;
-      { ProfScope ps(m, PK_QKV); launches += launch_gemv(g, EPI_STORE, ml, st); }
+      { ProfScope ps(m, PK_QKV); launches += project(m, g, EPI_STORE, ml); }
       { ProfScope ps(m, PK_ROPE);
         launches += launch_rope_append(m->qkv(), m->rope(), m->Kc, m->Vc, m->sched(), l, ROWS_PREFIX,
                                        0, ml, dm, st); }
@@ -224,25 +249,29 @@ static int32_t run_step(d3_model *m, const StepArgs &a, const int32_t *n, const 
                                      m->lay.max_splits, m->part_o(), m->part_ml(), m->attn_out(), dm, st); }
       // output projection + residual
       g.W = m->wo[l]; g.R = dm.d; g.K = nq; g.act = m->attn_out(); g.act_stride = nq;
+      g.tmap_w = tm ? &m->tm_o[l] : nullptr;
       g.gain = nullptr; g.out = m->x(); g.out_stride = dm.d;
-      { ProfScope ps(m, PK_OPROJ); launches += launch_gemv(g, EPI_RESID, ml, st); }
+      { ProfScope ps(m, PK_OPROJ); launches += project(m, g, EPI_RESID, ml); }
       // RMSNorm + gate/up + SiLU * mul
       g.W = m->w_gate[l]; g.W2 = m->w_up[l]; g.R = dm.f; g.K = dm.d; g.act = m->x();
+      g.tmap_w = tm ? &m->tm_gate[l] : nullptr; g.tmap_w2 = tm ? &m->tm_up[l] : nullptr;
       g.act_stride = dm.d; g.gain = m->mlp_norm[l]; g.out = m->u(); g.out_stride = dm.f;
-      { ProfScope ps(m, PK_GATEUP); launches += launch_gemv(g, EPI_SWIGLU, ml, st); }
+      { ProfScope ps(m, PK_GATEUP); launches += project(m, g, EPI_SWIGLU, ml); }
       // down projection + residual
       g.W = m->w_down[l]; g.W2 = nullptr; g.R = dm.d; g.K = dm.f; g.act = m->u();
+      g.tmap_w = tm ? &m->tm_down[l] : nullptr; g.tmap_w2 = nullptr;
       g.act_stride = dm.f; g.gain = nullptr; g.out = m->x(); g.out_stride = dm.d;
-      { ProfScope ps(m, PK_DOWN); launches += launch_gemv(g, EPI_RESID, ml, st); }
+      { ProfScope ps(m, PK_DOWN); launches += project(m, g, EPI_RESID, ml); }
     }
     if (c.kv_fill == D3_FILL_RECOMPUTE && ml < B) {
       // rows that drop block l: K,V from the block's own norm, W_k, W_v on the carried state
       g.row_mode = ROWS_SUFFIX;
       g.W = m->wqkv[l] + (size_t)nq * dm.d; g.W2 = nullptr; g.R = 2 * nkv; g.K = dm.d;
+      g.tmap_w = tm ? &m->tm_kv[l] : nullptr; g.tmap_w2 = nullptr;
       g.act = m->x(); g.act_stride = dm.d; g.gain = m->attn_norm[l];
       g.out = m->qkv(); g.out_stride = dm.qkv_rows; g.out_col0 = nq;
       ProfScope ps(m, PK_FILL);
-      launches += launch_gemv(g, EPI_STORE, B - ml, st);
+      launches += project(m, g, EPI_STORE, B - ml);
       launches += launch_rope_append(m->qkv(), m->rope(), m->Kc, m->Vc, m->sched(), l, ROWS_SUFFIX,
                                      1, B - ml, dm, st);
       g.out_col0 = 0;
@@ -256,8 +285,9 @@ static int32_t run_step(d3_model *m, const StepArgs &a, const int32_t *n, const 
   if (logits_dev) {
     g.layer = 0; g.row_mode = logits_mode;
     g.W = m->lm_head; g.W2 = nullptr; g.R = dm.V; g.K = dm.d; g.act = m->x(); g.act_stride = dm.d;
+    g.tmap_w = tm ? &m->tm_head : nullptr; g.tmap_w2 = nullptr;
     g.gain = m->final_norm; g.out = logits_dev; g.out_stride = dm.V; g.out_col0 = 0;
-    { ProfScope ps(m, PK_HEAD); launches += launch_gemv(g, EPI_LOGITS, logits_mode == ROWS_LAST ? 1 : B, st); }
+    { ProfScope ps(m, PK_HEAD); launches += project(m, g, EPI_LOGITS, logits_mode == ROWS_LAST ? 1 : B); }
   }
   m->last_B = B;
   for (int b = 0; b < B; ++b) m->last_perm[b] = perm[b];
@@ -403,6 +433,34 @@ int32_t d3_load(const d3_config *cfg, const d3_weights *w, void *kv_dev, void *s
   m->layer_bytes = 2 * ((int64_t)m->dm.qkv_rows * d + d * cfg->n_q_heads * cfg->head_dim + 3 * d * f + 2 * d);
   m->head_bytes = 2 * ((int64_t)cfg->vocab * d + d);
   if (init_kernel_attributes() != 0) { delete m; return D3_ECUDA; }
+  // tensor-core projections: usable when the driver encodes every weight's tensor map
+  m->tc.ok = tc_init() == 0;
+  m->tc.act_split = reinterpret_cast<bf16 *>(m->scratch + m->lay.act_split);
+  m->tc.act_bytes = m->lay.act_split_bytes;
+  m->tc.wait_ns = 2000000000ull;
+  {
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1)
+      sms = 148;
+    m->tc.sm_count = sms;
+  }
+  m->tm_ok = m->tc.ok;
+  if (m->tm_ok) {
+    const int nq = m->dm.Hq * m->dm.dh, nkv = m->dm.Hkv * m->dm.dh, dd = m->dm.d, ff = m->dm.f;
+    m->tm_qkv.resize(L); m->tm_kv.resize(L); m->tm_o.resize(L);
+    m->tm_gate.resize(L); m->tm_up.resize(L); m->tm_down.resize(L);
+    bool ok = tc_weight_map(&m->tm_head, m->lm_head, m->dm.V, dd);
+    for (int l = 0; l < L && ok; ++l) {
+      ok = tc_weight_map(&m->tm_qkv[l], m->wqkv[l], m->dm.qkv_rows, dd) &&
+           tc_weight_map(&m->tm_kv[l], m->wqkv[l] + (size_t)nq * dd, 2 * nkv, dd) &&
+           tc_weight_map(&m->tm_o[l], m->wo[l], dd, nq) &&
+           tc_weight_map(&m->tm_gate[l], m->w_gate[l], ff, dd) &&
+           tc_weight_map(&m->tm_up[l], m->w_up[l], ff, dd) &&
+           tc_weight_map(&m->tm_down[l], m->w_down[l], dd, ff);
+    }
+    m->tm_ok = ok;
+  }
   m->exec_mode = D3_EXEC_AUTO;
   for (int l = 0; l < L; ++l)
     m->layer_tab_host.push_back(LayerPtrs{m->attn_norm[l], m->wqkv[l], m->wo[l], m->mlp_norm[l],
@@ -587,7 +645,8 @@ int32_t d3_sync(d3_model *m) {
 }
 
 int32_t d3_set_exec(d3_model *m, int32_t mode) {
-  if (!m || (mode != D3_EXEC_AUTO && mode != D3_EXEC_KERNELS)) return D3_EINVAL;
+  if (!m || (mode != D3_EXEC_AUTO && mode != D3_EXEC_KERNELS && mode != D3_EXEC_TENSOR)) return D3_EINVAL;
+  if (mode == D3_EXEC_TENSOR && !m->tm_ok) return D3_EINVAL;
   m->exec_mode = mode;
   return D3_OK;
 }

@@ -5,6 +5,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <map>
+
 #include "d3.h"
 
 namespace d3 {
@@ -53,8 +55,14 @@ enum Epilogue {
   EPI_LOGITS = 3   // out[caller row][r] = y    (un-permuted)
 };
 
+// Opaque storage of one TMA tensor map (encoded on the host by the driver).
+struct alignas(64) TMap {
+  uint64_t w[16];
+};
+
 struct GemvArgs {
   const bf16 *W, *W2;   // [R][K] row-major (W2: second matrix of EPI_SWIGLU)
+  const TMap *tmap_w, *tmap_w2;  // host pointers, nullable: tensor maps of W and W2 (tensor-core path)
   int R, K;
   const float *act;     // [rows][act_stride]
   int act_stride;
@@ -104,9 +112,20 @@ struct FusedParams {
   unsigned long long wait_ns;   // bound of every device-side wait
 };
 
+// Host state of the tensor-core projection path.
+struct TcContext {
+  bool ok;                              // the driver's tensor-map encoder is there and the kernels are set up
+  bf16 *act_split;                      // device: activations as bf16 hi rows then lo rows, [2 NP][K]
+  size_t act_bytes;
+  std::map<uint64_t, TMap> act_maps;    // tensor maps of act_split, keyed by (NP, K)
+  int sm_count;
+  unsigned long long wait_ns;           // bound of every device-side wait
+};
+
 // Byte offsets of the regions of the caller's scratch buffer.
 struct Layout {
-  size_t sched, rope, x, qkv, attn_out, part_o, part_ml, u, layer_tab, bar, phase, part_fused, total;
+  size_t sched, rope, x, qkv, attn_out, part_o, part_ml, u, layer_tab, bar, phase, part_fused, act_split,
+      act_split_bytes, total;
   int max_splits;
 };
 
@@ -129,6 +148,11 @@ int launch_attention(const float *qkv, const bf16 *Kc, const bf16 *Vc, const Dev
 int launch_fill_copy(bf16 *Kc, bf16 *Vc, const DevSched *s, int B, const Dims &dm, cudaStream_t st);
 int launch_argmax(const float *logits, int B, int V, int32_t *out, cudaStream_t st);
 int init_kernel_attributes();
+// tensor-core projections: 0 when the path is usable on this device / driver
+int tc_init();
+bool tc_weight_map(TMap *out, const bf16 *W, int R, int K);
+// pre-pass + GEMM for m_rows rows; returns kernels launched, 0 = not served (use launch_gemv)
+int launch_gemm_tc(TcContext &tc, const GemvArgs &g, int epi, int m_rows, cudaStream_t st);
 // fused batch-1 step: returns 1 and the launch plan when the kernel serves `c` on this device
 int fused_plan(const d3_config &c, int *grid, int *n_stages, int *act_floats, size_t *smem, void **func);
 int launch_fused_step(void *func, int grid, size_t smem, FusedParams &fp, cudaStream_t st);
