@@ -176,7 +176,7 @@ int32_t d3_read_kv(d3_model *m, int32_t layer, int32_t slot, int32_t pos, float 
 #define D3_EXEC_AUTO 0
 #define D3_EXEC_KERNELS 1
 #define D3_EXEC_TENSOR 2
-#define D3_TENSOR_MIN_ROWS 5
+#define D3_TENSOR_MIN_ROWS 2
 int32_t d3_set_exec(d3_model *m, int32_t mode);
 
 /* Per-kernel-class device times (measurement aid for Sec. 4.2-style wall-clock
