@@ -179,7 +179,10 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int kb0 = blockIdx.y * t.kb_per_split;
   const int kb1 = min(t.n_kb, kb0 + t.kb_per_split);
-  if (kb0 >= kb1) return;   // uniform over the CTA; the host launches no such slice
+  if (kb0 >= kb1) {         // uniform over the CTA; the host launches no such slice
+    pdl_wait();
+    return;
+  }
   const int n_it = kb1 - kb0;
   const int S = t.n_stages;
   const int N = 2 * t.NP;
@@ -208,6 +211,10 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
   __syncthreads();
   fence_after_sync();
   const uint32_t tmem = s_tmem;
+  pdl_trigger();
+  // Up to here nothing depends on an earlier kernel.  The producer lane goes one step further: the
+  // weights are constants, so it puts the first ring fill of weight tiles in flight before it waits.
+  if (!(warp == 0 && lane == 0)) pdl_wait();
 
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
@@ -216,14 +223,28 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
       if (EPI == EPI_SWIGLU) { row_a = blockIdx.x * kBoxRows; row_b = row_a; }
       else { row_a = blockIdx.x * kTileM; row_b = row_a + kBoxRows; }
       int issued = 0;
-      for (int it = 0; it < n_it; ++it) {
+      const int first = min(S, n_it);
+      for (int it = 0; it < first; ++it) {   // first fill: weight tiles only
+        const uint32_t full = smem_addr(&s_full[it]);
+        const uint32_t a = ring + (uint32_t)it * stage_bytes;
+        const int x = (kb0 + it) * kTileK;   // x * 2 bytes is a multiple of 128
+        bar_expect_tx(full, stage_bytes);
+        tma_load_2d(a, &map_w0, x, row_a, full);
+        tma_load_2d(a + kBoxRows * kTileK * 2, &map_w1, x, row_b, full);
+      }
+      pdl_wait();                            // the activations come from the previous kernel
+      for (int it = 0; it < first; ++it) {
+        const uint32_t a = ring + (uint32_t)it * stage_bytes;
+        tma_load_2d(a + kABytes, &map_act, (kb0 + it) * kTileK, 0, smem_addr(&s_full[it]));
+        issued = it + 1;
+      }
+      for (int it = first; it < n_it; ++it) {
         const int s = it % S, fill = it / S;
-        if (fill > 0 &&
-            !bar_wait(smem_addr(&s_empty[s]), (uint32_t)((fill - 1) & 1), abort_flag, t.wait_ns, true))
+        if (!bar_wait(smem_addr(&s_empty[s]), (uint32_t)((fill - 1) & 1), abort_flag, t.wait_ns, true))
           break;
         const uint32_t full = smem_addr(&s_full[s]);
         const uint32_t a = ring + (uint32_t)s * stage_bytes;
-        const int x = (kb0 + it) * kTileK;   // x * 2 bytes is a multiple of 128
+        const int x = (kb0 + it) * kTileK;
         bar_expect_tx(full, stage_bytes);
         tma_load_2d(a, &map_w0, x, row_a, full);
         tma_load_2d(a + kBoxRows * kTileK * 2, &map_w1, x, row_b, full);
@@ -345,10 +366,14 @@ struct SplitArgs {
   int layer, row_mode;
 };
 
+// grid (rows, K / 1024 chunks): every CTA of a row recomputes the row's sum of squares (a few
+// KB out of L2) and converts its own 1024-element chunk.
 __global__ void __launch_bounds__(256) k_act_split(const SplitArgs a) {
   __shared__ float s_red[8];
   __shared__ float s_scale;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  pdl_wait();
+  pdl_trigger();
   int r0, r1;
   row_span(a.sched, a.layer, a.row_mode, r0, r1);
   const int j = blockIdx.x, row = r0 + j;
@@ -374,7 +399,8 @@ __global__ void __launch_bounds__(256) k_act_split(const SplitArgs a) {
     sc = s_scale;
   }
   bf16 *hi = a.dst + (size_t)j * a.K, *lo = a.dst + (size_t)(a.NP + j) * a.K;
-  for (int k = tid * 4; k < a.K; k += 256 * 4) {
+  const int k = blockIdx.y * 1024 + tid * 4;
+  if (k < a.K) {
     float4 v = *reinterpret_cast<const float4 *>(src + k);
     if (a.gain) {
       uint2 gw = *reinterpret_cast<const uint2 *>(a.gain + k);
@@ -393,7 +419,7 @@ __global__ void __launch_bounds__(256) k_act_split(const SplitArgs a) {
   }
   if (a.zero_out) {
     float *o = a.zero_out + (size_t)row * a.out_stride + a.out_col0;
-    for (int c = tid; c < a.R; c += 256) o[c] = 0.f;
+    for (int c = blockIdx.y * 256 + tid; c < a.R; c += gridDim.y * 256) o[c] = 0.f;
   }
 }
 
@@ -471,8 +497,8 @@ int launch_gemm_tc(TcContext &tc, const GemvArgs &g, int epi, int m_rows, cudaSt
   const int n_kb = (g.K + kTileK - 1) / kTileK;
   int ksplit = 1;
   if (epi == EPI_STORE || epi == EPI_RESID) {
-    // aim at two resident CTAs per SM, slices of at least 8 k-blocks
-    ksplit = (2 * tc.sm_count + tiles - 1) / tiles;
+    // all CTAs resident at once (two per SM), slices of at least 8 k-blocks
+    ksplit = 2 * tc.sm_count / tiles;
     if (ksplit > n_kb / 8) ksplit = n_kb / 8;
     if (ksplit < 1) ksplit = 1;
     if (ksplit > 16) ksplit = 16;
@@ -486,7 +512,7 @@ int launch_gemm_tc(TcContext &tc, const GemvArgs &g, int epi, int m_rows, cudaSt
   sa.zero_out = (epi == EPI_STORE && ksplit > 1) ? g.out : nullptr;
   sa.out_stride = g.out_stride; sa.out_col0 = g.out_col0; sa.R = g.R;
   sa.sched = g.sched; sa.layer = g.layer; sa.row_mode = g.row_mode;
-  k_act_split<<<m_rows, 256, 0, st>>>(sa);
+  launch_pdl(k_act_split, dim3(m_rows, (g.K + 1023) / 1024), dim3(256), 0, st, sa);
 
   TcArgs t;
   t.R = g.R; t.K = g.K; t.NP = NP; t.n_kb = n_kb; t.kb_per_split = per;
@@ -506,10 +532,10 @@ int launch_gemm_tc(TcContext &tc, const GemvArgs &g, int epi, int m_rows, cudaSt
   const CUtensorMap *ma = reinterpret_cast<const CUtensorMap *>(&it->second);
   dim3 grid((unsigned)tiles, (unsigned)ksplit);
   switch (epi) {
-    case EPI_STORE: k_gemm_tc<EPI_STORE><<<grid, kTcThreads, smem, st>>>(*w0, *w1, *ma, t); break;
-    case EPI_RESID: k_gemm_tc<EPI_RESID><<<grid, kTcThreads, smem, st>>>(*w0, *w1, *ma, t); break;
-    case EPI_SWIGLU: k_gemm_tc<EPI_SWIGLU><<<grid, kTcThreads, smem, st>>>(*w0, *w1, *ma, t); break;
-    default: k_gemm_tc<EPI_LOGITS><<<grid, kTcThreads, smem, st>>>(*w0, *w1, *ma, t); break;
+    case EPI_STORE: launch_pdl(k_gemm_tc<EPI_STORE>, grid, dim3(kTcThreads), smem, st, *w0, *w1, *ma, t); break;
+    case EPI_RESID: launch_pdl(k_gemm_tc<EPI_RESID>, grid, dim3(kTcThreads), smem, st, *w0, *w1, *ma, t); break;
+    case EPI_SWIGLU: launch_pdl(k_gemm_tc<EPI_SWIGLU>, grid, dim3(kTcThreads), smem, st, *w0, *w1, *ma, t); break;
+    default: launch_pdl(k_gemm_tc<EPI_LOGITS>, grid, dim3(kTcThreads), smem, st, *w0, *w1, *ma, t); break;
   }
   return 2;
 }

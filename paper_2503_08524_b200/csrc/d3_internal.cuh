@@ -4,6 +4,7 @@
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
+#include <string.h>
 
 #include <map>
 
@@ -128,6 +129,36 @@ struct Layout {
       act_split_bytes, total;
   int max_splits;
 };
+
+// Programmatic dependent launch: every kernel of the step sequence is launched
+// with the stream-serialization attribute, so that it may become resident while
+// its predecessor still runs.  EVERY thread calls pdl_wait() before it touches
+// anything another kernel of the stream writes or reads (it returns once all
+// earlier kernels have completed and their writes are visible); what precedes
+// the call may only touch kernel parameters, constant weights and the CTA's own
+// shared / tensor memory.  Because no CTA exits without the wait, completion of
+// a kernel implies completion of all its predecessors.
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                              Args... args) {
+  cudaLaunchConfig_t cfg;
+  memset(&cfg, 0, sizeof(cfg));
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+#endif
 
 Layout make_layout(const d3_config &c);
 bool config_ok(const d3_config *c);

@@ -61,6 +61,8 @@ k_schedule_embed(const __grid_constant__ StepArgs a, DevSched *s, const bf16 *E,
   __shared__ int sn[D3_MAX_BATCH], slo[D3_MAX_BATCH], shi[D3_MAX_BATCH], sperm[D3_MAX_BATCH];
   __shared__ int sm[D3_MAX_LAYERS];
   const int B = a.B, L = a.L, tid = threadIdx.x;
+  pdl_wait();
+  pdl_trigger();
   if (tid < B) {
     int i = a.gi[tid], n = 0;
     for (int k = 1; k <= L; ++k) n += (i < a.thr[k]) ? 1 : 0;
@@ -116,7 +118,7 @@ k_schedule_embed(const __grid_constant__ StepArgs a, DevSched *s, const bf16 *E,
 
 int launch_schedule_embed(const StepArgs &a, DevSched *s, const bf16 *E, float *x, int d,
                           cudaStream_t st) {
-  k_schedule_embed<<<a.B, kThreads, 0, st>>>(a, s, E, x, d);
+  launch_pdl(k_schedule_embed, dim3(a.B), dim3(kThreads), 0, st, a, s, E, x, d);
   return 1;
 }
 
@@ -138,6 +140,8 @@ k_gemv(const GemvArgs g, int kc_max) {
   __shared__ float s_red[kWarps][MT];
   __shared__ float s_scale[MT];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  pdl_wait();
+  pdl_trigger();
   int r0, r1;
   row_range(g.sched, g.layer, g.row_mode, r0, r1);
   if (r0 >= r1) return;
@@ -294,7 +298,7 @@ static void gemv_launch(const GemvArgs &g, cudaStream_t st) {
   int kpad = (g.K + 255) / 256 * 256;
   if (kc_max > kpad) kc_max = kpad;
   size_t smem = (size_t)MT * kc_max * 4;
-  k_gemv<MT, EPI><<<grid, kThreads, smem, st>>>(g, kc_max);
+  launch_pdl(k_gemv<MT, EPI>, dim3(grid), dim3(kThreads), smem, st, g, kc_max);
 }
 
 template <int EPI>
@@ -334,46 +338,48 @@ int init_kernel_attributes() {
 // ---------------------------------------------------------- RoPE + KV append
 // Rotates q (in place, fp32) and k at the row's position, pair (j, j + dh/2),
 // and stores k, v as bf16 at cache[layer][slot][kv head][pos][:].
+// grid (rows, head chunks): a thread owns one pair of one head; the heads are
+// numbered q heads, then k heads, then v heads.
 __global__ void __launch_bounds__(kThreads)
 k_rope_append(float *qkv, const float2 *rope, bf16 *Kc, bf16 *Vc, const DevSched *s, int layer,
               int row_mode, int kv_only, Dims dm) {
+  pdl_wait();
+  pdl_trigger();
   int r0, r1;
   row_range(s, layer, row_mode, r0, r1);
   const int row = r0 + blockIdx.x;
   if (row >= r1) return;
-  const int dh = dm.dh, half = dh / 2, nq = dm.Hq * dh, nkv = dm.Hkv * dh;
+  const int dh = dm.dh, half = dh / 2;
+  const int hs = blockIdx.y * (kThreads / half) + threadIdx.x / half, j = threadIdx.x % half;
+  if (hs >= dm.Hq + 2 * dm.Hkv) return;
   const int pos = s->pos_s[row], slot = s->slot_s[row];
-  float *q = qkv + (size_t)row * dm.qkv_rows;
-  float *k = q + nq, *v = k + nkv;
-  const float2 *tab = rope + (size_t)pos * half;
+  float *p = qkv + (size_t)row * dm.qkv_rows + (size_t)hs * dh;
   const size_t cbase = ((size_t)layer * dm.max_slots + slot) * dm.Hkv;
-  if (!kv_only) {
-    for (int i = threadIdx.x; i < dm.Hq * half; i += kThreads) {
-      int h = i / half, j = i % half;
-      float2 cs = tab[j];
-      float a = q[h * dh + j], b = q[h * dh + j + half];
-      q[h * dh + j] = a * cs.x - b * cs.y;
-      q[h * dh + j + half] = a * cs.y + b * cs.x;
-    }
-  }
-  for (int i = threadIdx.x; i < dm.Hkv * half; i += kThreads) {
-    int h = i / half, j = i % half;
-    float2 cs = tab[j];
-    float a = k[h * dh + j], b = k[h * dh + j + half];
-    bf16 *dst = Kc + ((cbase + h) * dm.max_seq + pos) * dh;
+  if (hs < dm.Hq) {
+    if (kv_only) return;
+    const float2 cs = rope[(size_t)pos * half + j];
+    const float a = p[j], b = p[j + half];
+    p[j] = a * cs.x - b * cs.y;
+    p[j + half] = a * cs.y + b * cs.x;
+  } else if (hs < dm.Hq + dm.Hkv) {
+    const float2 cs = rope[(size_t)pos * half + j];
+    const float a = p[j], b = p[j + half];
+    bf16 *dst = Kc + ((cbase + (hs - dm.Hq)) * dm.max_seq + pos) * dh;
     dst[j] = __float2bfloat16_rn(a * cs.x - b * cs.y);
     dst[j + half] = __float2bfloat16_rn(a * cs.y + b * cs.x);
-  }
-  for (int i = threadIdx.x; i < nkv; i += kThreads) {
-    int h = i / dh, e = i % dh;
-    Vc[((cbase + h) * dm.max_seq + pos) * dh + e] = __float2bfloat16_rn(v[i]);
+  } else {
+    bf16 *dst = Vc + ((cbase + (hs - dm.Hq - dm.Hkv)) * dm.max_seq + pos) * dh;
+    dst[j] = __float2bfloat16_rn(p[j]);
+    dst[j + half] = __float2bfloat16_rn(p[j + half]);
   }
 }
 
 int launch_rope_append(float *qkv, const float2 *rope, bf16 *Kc, bf16 *Vc, const DevSched *s,
                        int layer, int row_mode, int kv_only, int m_rows, const Dims &dm,
                        cudaStream_t st) {
-  k_rope_append<<<m_rows, kThreads, 0, st>>>(qkv, rope, Kc, Vc, s, layer, row_mode, kv_only, dm);
+  const int heads_per_cta = kThreads / (dm.dh / 2);
+  dim3 grid(m_rows, (dm.Hq + 2 * dm.Hkv + heads_per_cta - 1) / heads_per_cta);
+  launch_pdl(k_rope_append, grid, dim3(kThreads), 0, st, qkv, rope, Kc, Vc, s, layer, row_mode, kv_only, dm);
   return 1;
 }
 
@@ -389,6 +395,8 @@ __global__ void __launch_bounds__(kThreads)
 k_attn_partial(const float *qkv, const bf16 *Kc, const bf16 *Vc, const DevSched *s, int layer,
                int split_len, int max_splits, float *part_o, float *part_ml, Dims dm) {
   constexpr int EPL = DH / 8;
+  pdl_wait();
+  pdl_trigger();
   const int row = blockIdx.z;
   if (row >= s->m[layer]) return;
   const int len = s->pos_s[row] + 1;
@@ -508,6 +516,8 @@ k_attn_partial(const float *qkv, const bf16 *Kc, const bf16 *Vc, const DevSched 
 // merge the splits of one (row, head): attn_out[row][h*dh + e]
 __global__ void k_attn_combine(const float *part_o, const float *part_ml, const DevSched *s, int layer,
                                int split_len, int max_splits, float *attn_out, Dims dm) {
+  pdl_wait();
+  pdl_trigger();
   const int row = blockIdx.y, h = blockIdx.x, e = threadIdx.x;
   if (row >= s->m[layer]) return;
   const int len = s->pos_s[row] + 1;
@@ -531,16 +541,16 @@ static void attn_launch(const float *qkv, const bf16 *Kc, const bf16 *Vc, const 
   int G = dm.Hq / dm.Hkv;
   if (G % 4 == 0) {
     dim3 grid(n_splits, dm.Hq / 4, m_rows);
-    k_attn_partial<DH, 4><<<grid, kThreads, 0, st>>>(qkv, Kc, Vc, s, layer, split_len, max_splits,
-                                                     part_o, part_ml, dm);
+    launch_pdl(k_attn_partial<DH, 4>, grid, dim3(kThreads), 0, st, qkv, Kc, Vc, s, layer, split_len,
+               max_splits, part_o, part_ml, dm);
   } else if (G % 2 == 0) {
     dim3 grid(n_splits, dm.Hq / 2, m_rows);
-    k_attn_partial<DH, 2><<<grid, kThreads, 0, st>>>(qkv, Kc, Vc, s, layer, split_len, max_splits,
-                                                     part_o, part_ml, dm);
+    launch_pdl(k_attn_partial<DH, 2>, grid, dim3(kThreads), 0, st, qkv, Kc, Vc, s, layer, split_len,
+               max_splits, part_o, part_ml, dm);
   } else {
     dim3 grid(n_splits, dm.Hq, m_rows);
-    k_attn_partial<DH, 1><<<grid, kThreads, 0, st>>>(qkv, Kc, Vc, s, layer, split_len, max_splits,
-                                                     part_o, part_ml, dm);
+    launch_pdl(k_attn_partial<DH, 1>, grid, dim3(kThreads), 0, st, qkv, Kc, Vc, s, layer, split_len,
+               max_splits, part_o, part_ml, dm);
   }
 }
 
@@ -554,7 +564,8 @@ int launch_attention(const float *qkv, const bf16 *Kc, const bf16 *Vc, const Dev
   else
     attn_launch<32>(qkv, Kc, Vc, s, layer, m_rows, split_len, n_splits, max_splits, part_o, part_ml, dm, st);
   dim3 cgrid(dm.Hq, m_rows);
-  k_attn_combine<<<cgrid, dm.dh, 0, st>>>(part_o, part_ml, s, layer, split_len, max_splits, attn_out, dm);
+  launch_pdl(k_attn_combine, cgrid, dim3(dm.dh), 0, st, part_o, part_ml, s, layer, split_len, max_splits,
+             attn_out, dm);
   return 2;
 }
 
@@ -563,6 +574,8 @@ int launch_attention(const float *qkv, const bf16 *Kc, const bf16 *Vc, const Dev
 // of block lo-1 written earlier in this step, or zeros when the window opens at
 // block 0.  grid (L, B).
 __global__ void k_fill_copy(bf16 *Kc, bf16 *Vc, const DevSched *s, Dims dm) {
+  pdl_wait();
+  pdl_trigger();
   const int l = blockIdx.x, row = blockIdx.y;
   const int lo = s->lo_s[row], hi = s->hi_s[row];
   if (l < lo || l >= hi) return;
@@ -584,12 +597,14 @@ __global__ void k_fill_copy(bf16 *Kc, bf16 *Vc, const DevSched *s, Dims dm) {
 
 int launch_fill_copy(bf16 *Kc, bf16 *Vc, const DevSched *s, int B, const Dims &dm, cudaStream_t st) {
   dim3 grid(dm.L, B);
-  k_fill_copy<<<grid, 128, 0, st>>>(Kc, Vc, s, dm);
+  launch_pdl(k_fill_copy, grid, dim3(128), 0, st, Kc, Vc, s, dm);
   return 1;
 }
 
 // --------------------------------------------------------------------- argmax
 __global__ void __launch_bounds__(1024) k_argmax(const float *logits, int V, int32_t *out) {
+  pdl_wait();
+  pdl_trigger();
   const float *p = logits + (size_t)blockIdx.x * V;
   float best = -INFINITY;
   int bi = 0x7fffffff;
@@ -615,7 +630,7 @@ __global__ void __launch_bounds__(1024) k_argmax(const float *logits, int V, int
 }
 
 int launch_argmax(const float *logits, int B, int V, int32_t *out, cudaStream_t st) {
-  k_argmax<<<B, 1024, 0, st>>>(logits, V, out);
+  launch_pdl(k_argmax, dim3(B), dim3(1024), 0, st, logits, V, out);
   return 1;
 }
 
