@@ -71,7 +71,7 @@ def test_schedule_kernel_large_L(B):
 @pytest.mark.parametrize("shape", [I.TINY, I.TINY_GQA], ids=["mha", "gqa"])
 @pytest.mark.parametrize("alpha", [1.0, 0.98, 0.95])
 @pytest.mark.parametrize("kv_round", [False, True], ids=["kv-exact", "kv-bf16"])
-@pytest.mark.parametrize("exec_mode", [0, 1], ids=["fused", "kernels"])
+@pytest.mark.parametrize("exec_mode", [0, 1, 2], ids=["fused", "kernels", "tensor"])
 def test_tiny_generate_teacher_forced(B, shape, alpha, kv_round, exec_mode):
     orc, gpu = make_pair(shape, SEED, 2, 64, 1, start_id=0, kv_round_bf16=kv_round)
     gpu.d3_set_exec(exec_mode)
@@ -126,10 +126,14 @@ def test_tiny_greedy_tokens_identical(B):
 
 @pytest.mark.parametrize("anchor,start", [(0, 0), (0, 1), (0, 2), (1, 0)])
 @pytest.mark.parametrize("fill", [0, 1, 2])
-def test_batched_mixed_depth_steps(B, anchor, start, fill):
+@pytest.mark.parametrize("exec_mode", [0, 1], ids=["tensor-cores", "fma"])
+def test_batched_mixed_depth_steps(B, anchor, start, fill, exec_mode):
+    # exec 0: depth groups of 2+ rows project on the tensor cores, single rows by FMA GEMV;
+    # exec 1: FMA GEMVs throughout
     shape = I.TINY_GQA
     Bn, alpha = 7, 0.96
     orc, gpu = make_pair(shape, SEED + 2, 8, 96, 8, start_id=start, anchor=anchor, kv_fill=fill)
+    gpu.d3_set_exec(exec_mode)
     gpu.poison_kv()
     orc.poison_kv()
     lens = I.uniform_ints(SEED + 2, 77, Bn, 3, 40)
@@ -237,14 +241,16 @@ def test_prefill_longer_than_a_batch_and_ragged_lengths(B):
 # ----------------------------------------------------------- production widths
 
 @pytest.mark.parametrize("base,layers,Bn", [(I.LLAMA_7B, 3, 1), (I.LLAMA_7B, 2, 5), (I.LLAMA_70B, 2, 3),
-                                            (I.LLAMA_13B, 2, 1), (I.LLAMA_70B, 2, 1)],
+                                            (I.LLAMA_13B, 2, 1), (I.LLAMA_70B, 2, 1), (I.LLAMA_7B, 2, 32),
+                                            (I.LLAMA_13B, 2, 8), (I.LLAMA_70B, 2, 4)],
                          ids=["7b-width-b1", "7b-width-b5", "70b-width-gqa-b3", "13b-width-b1",
-                              "70b-width-gqa-b1"])
+                              "70b-width-gqa-b1", "7b-width-b32", "13b-width-b8", "70b-width-gqa-b4"])
 def test_production_widths(B, base, layers, Bn):
-    # full-width blocks (same kernel shapes and tiling as the benchmark), few layers
+    # full-width blocks (same kernel shapes and tiling as the benchmark), few layers;
+    # batches of 2+ rows take the tensor-core projections, single rows the fused step
     shape = base.with_layers(layers)
-    orc, gpu = make_pair(shape, SEED + 5, Bn, 96, 8, start_id=1, gain_jitter=0.1)
-    lens = I.uniform_ints(SEED + 5, 3, Bn, 5, 40)
+    orc, gpu = make_pair(shape, SEED + 5, Bn, 96, max(8, Bn), start_id=1, gain_jitter=0.1)
+    lens = I.uniform_ints(SEED + 5, 3, Bn, 5, 40 if Bn <= 8 else 12)
     for b in range(Bn):
         p = I.prompt_tokens(shape, SEED + 5, b, lens[b]).numpy()
         o = orc.prefill(b, p)
