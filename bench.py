@@ -369,9 +369,10 @@ def main():
         oshape, scale, note = oracle_shape_and_scale(shape)
         w_cpu = I.weights_to({k: (v[:oshape.n_layers] if isinstance(v, list) else v)
                               for k, v in w.items()}, "cpu")
-        tps, dt, cores = time_oracle(oshape, w_cpu, args.alpha, start_id, 16, 1)
+        osteps = 96 if scale == 1.0 else 192      # ~15 s of CPU work on the box's 16 cores
+        tps, dt, cores = time_oracle(oshape, w_cpu, args.alpha, start_id, osteps, 1)
         cpu_baseline = {"value": tps * scale, "unit": "tokens/s", "cores": cores, "kind": "oracle",
-                        "sample": f"fp64 C oracle, 7B shape, {note}, prompt {ORACLE_PROMPT}, 16 decode "
+                        "sample": f"fp64 C oracle, 7B shape, {note}, prompt {ORACLE_PROMPT}, {osteps} decode "
                                   f"steps at alpha={args.alpha}, {dt:.1f} s of CPU work"}
 
     line = {
