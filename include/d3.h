@@ -54,6 +54,18 @@ extern "C" {
                                to the carried hidden state                            */
 
 #define D3_KV_CONTIGUOUS 0  /* K then V, each [L][slot][Hkv][max_seq][head_dim] bf16  */
+#define D3_KV_PAGED 1       /* K then V, each a pool [n_pages][Hkv][page_size][head_dim] bf16.
+                               A page holds page_size consecutive positions of ONE sequence
+                               in ONE block; the library hands pages out on demand (host
+                               bookkeeping, a device table [L][slot][max_seq / page_size]) and
+                               takes them back in d3_reset_slot.  Depth-aware: with
+                               D3_FILL_NONE a (token, block) pair inside the token's dropped
+                               window is never written, so no page is taken for a block once
+                               the sequence's tokens stop running it (Sec. 3.2 leaves those
+                               states undefined; nothing reads them while depth only decays).
+                               Page 0 is reserved and zero-filled by d3_load: it stands in
+                               for every page never written.  Decode steps of a paged model
+                               always run as the sequence of kernels.                       */
 
 typedef struct d3_config {
   uint32_t struct_size;     /* sizeof(d3_config), checked                              */
@@ -72,7 +84,11 @@ typedef struct d3_config {
   int32_t start_id;         /* 0..L: first droppable block, 0-based (floor(start * L)) */
   int32_t anchor;           /* D3_ANCHOR_*                                             */
   int32_t kv_fill;          /* D3_FILL_*                                               */
-  int32_t kv_layout;        /* D3_KV_CONTIGUOUS                                        */
+  int32_t kv_layout;        /* D3_KV_CONTIGUOUS or D3_KV_PAGED                         */
+  int32_t page_size;        /* PAGED: positions per page, a power of two 16..1024 that
+                               divides max_seq; CONTIGUOUS: 0                          */
+  int32_t n_pages;          /* PAGED: pages in the pool (page 0 reserved), >= 2;
+                               CONTIGUOUS: 0                                           */
 } d3_config;
 
 /* DEVICE pointers to bf16 tensors; the per-layer members are HOST arrays of L
@@ -242,6 +258,9 @@ int32_t d3_decode_step_noalloc(const d3_config *cfg, const d3_weights *weights, 
                                double alpha, float *logits_dev, void *cuda_stream);
 
 int32_t d3_slot_pos(const d3_model *m, int32_t slot); /* tokens cached; D3_ESTATE if never prefilled */
+/* PAGED layout: pages handed out at the moment (the reserved page not counted);
+ * D3_EINVAL for a contiguous model.  Host bookkeeping only. */
+int32_t d3_kv_pages_used(const d3_model *m);
 int32_t d3_reset_slot(d3_model *m, int32_t slot);
 int32_t d3_sync(d3_model *m); /* wait for the stream; returns a deferred device status */
 void d3_free(d3_model *m);    /* host bookkeeping only */

@@ -20,10 +20,12 @@ ANCHOR_START, ANCHOR_TAIL = 0, 1
 FILL_NONE, FILL_COPY, FILL_RECOMPUTE = 0, 1, 2
 MAX_BATCH, MAX_LAYERS, PROF_KINDS = 64, 128, 22
 EXEC_AUTO, EXEC_KERNELS, EXEC_TENSOR = 0, 1, 2
+KV_CONTIGUOUS, KV_PAGED = 0, 1
 
 EXPORTS = ("d3_depth", "d3_schedule", "d3_workspace_bytes", "d3_load", "d3_prefill",
            "d3_decode_step", "d3_argmax", "d3_read_schedule", "d3_read_hidden", "d3_read_kv",
-           "d3_set_exec", "d3_profile", "d3_read_profile", "d3_profile_name", "d3_read_fused_phases", "d3_decode_step_noalloc", "d3_slot_pos", "d3_reset_slot", "d3_sync", "d3_free", "d3_strerror")
+           "d3_set_exec", "d3_profile", "d3_read_profile", "d3_profile_name", "d3_read_fused_phases", "d3_decode_step_noalloc", "d3_slot_pos",
+           "d3_kv_pages_used", "d3_reset_slot", "d3_sync", "d3_free", "d3_strerror")
 
 
 class Config(C.Structure):
@@ -32,7 +34,7 @@ class Config(C.Structure):
                                   "d_ffn", "vocab")] + \
         [("rms_eps", C.c_float), ("rope_base", C.c_float)] + \
         [(n, C.c_int32) for n in ("max_slots", "max_seq", "max_batch", "start_id", "anchor",
-                                  "kv_fill", "kv_layout")]
+                                  "kv_fill", "kv_layout", "page_size", "n_pages")]
 
 
 _PP = C.POINTER(C.c_void_p)
@@ -79,6 +81,7 @@ def _load() -> C.CDLL:
     lib.d3_decode_step_noalloc.argtypes = [C.POINTER(Config), C.POINTER(Weights), P, I32, I32, I32, I32,
                                            C.c_double, P, P]
     lib.d3_slot_pos.argtypes = [P, I32]
+    lib.d3_kv_pages_used.argtypes = [P]
     lib.d3_reset_slot.argtypes = [P, I32]
     lib.d3_sync.argtypes = [P]
     lib.d3_free.argtypes = [P]
@@ -117,10 +120,13 @@ def d3_schedule(L: int, alpha: float, start_id: int, anchor: int, gen_index: Seq
 
 
 def make_config(shape, max_slots: int, max_seq: int, max_batch: int, start_id: int = 0,
-                anchor: int = ANCHOR_START, kv_fill: int = FILL_COPY) -> Config:
+                anchor: int = ANCHOR_START, kv_fill: int = FILL_COPY, page_size: int = 0,
+                n_pages: int = 0) -> Config:
+    """page_size > 0 selects the paged KV layout with a pool of n_pages pages."""
     return Config(C.sizeof(Config), shape.n_layers, shape.d_model, shape.n_q_heads, shape.n_kv_heads,
                   shape.head_dim, shape.d_ffn, shape.vocab, shape.rms_eps, shape.rope_base,
-                  max_slots, max_seq, max_batch, start_id, anchor, kv_fill, 0)
+                  max_slots, max_seq, max_batch, start_id, anchor, kv_fill,
+                  KV_PAGED if page_size > 0 else KV_CONTIGUOUS, page_size, n_pages)
 
 
 def d3_workspace_bytes(cfg: Config):
@@ -164,10 +170,12 @@ class D3Model:
 
     def __init__(self, shape, weights: Dict[str, object], max_slots: int, max_seq: int,
                  max_batch: int = 1, start_id: int = 0, anchor: int = ANCHOR_START,
-                 kv_fill: int = FILL_COPY, device="cuda:0", stream: Optional[torch.cuda.Stream] = None):
+                 kv_fill: int = FILL_COPY, device="cuda:0", stream: Optional[torch.cuda.Stream] = None,
+                 page_size: int = 0, n_pages: int = 0):
         self.shape = shape
         self.device = torch.device(device)
-        self.cfg = make_config(shape, max_slots, max_seq, max_batch, start_id, anchor, kv_fill)
+        self.cfg = make_config(shape, max_slots, max_seq, max_batch, start_id, anchor, kv_fill,
+                               page_size, n_pages)
         kv_bytes, scratch_bytes = d3_workspace_bytes(self.cfg)
         self.kv_bytes, self.scratch_bytes = kv_bytes, scratch_bytes
         self.w = weights
@@ -309,6 +317,12 @@ class D3Model:
 
     def d3_slot_pos(self, slot: int) -> int:
         return int(LIB.d3_slot_pos(self.h, slot))
+
+    def d3_kv_pages_used(self) -> int:
+        rc = int(LIB.d3_kv_pages_used(self.h))
+        if rc < 0:
+            raise D3Error(rc, "d3_kv_pages_used")
+        return rc
 
     def d3_reset_slot(self, slot: int) -> None:
         rc = LIB.d3_reset_slot(self.h, slot)

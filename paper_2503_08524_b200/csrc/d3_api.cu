@@ -39,6 +39,9 @@ Layout make_layout(const d3_config &c) {
   y.act_split = off = align_up(off, 1024);
   y.act_split_bytes = 2 * ((B + 7) / 8 * 8) * kmax * sizeof(bf16);
   off = align_up(off + y.act_split_bytes, 256);
+  y.block_table = off;
+  if (c.kv_layout == D3_KV_PAGED)
+    off = align_up(off + (size_t)c.n_layers * c.max_slots * (c.max_seq / c.page_size) * sizeof(int32_t), 256);
   y.total = off;
   return y;
 }
@@ -56,7 +59,14 @@ bool config_ok(const d3_config *c) {
   if (c->start_id < 0 || c->start_id > c->n_layers) return false;
   if (c->anchor != D3_ANCHOR_START && c->anchor != D3_ANCHOR_TAIL) return false;
   if (c->kv_fill < D3_FILL_NONE || c->kv_fill > D3_FILL_RECOMPUTE) return false;
-  if (c->kv_layout != D3_KV_CONTIGUOUS) return false;
+  if (c->kv_layout == D3_KV_CONTIGUOUS) {
+    if (c->page_size != 0 || c->n_pages != 0) return false;
+  } else if (c->kv_layout == D3_KV_PAGED) {
+    const int ps = c->page_size;
+    if (ps < 16 || ps > 1024 || (ps & (ps - 1)) || c->max_seq % ps || c->n_pages < 2) return false;
+  } else {
+    return false;
+  }
   return true;
 }
 
@@ -117,6 +127,10 @@ struct d3_model {
   std::vector<TMap> tm_qkv, tm_kv, tm_o, tm_gate, tm_up, tm_down;
   TMap tm_head;
   bool tm_ok;
+  // paged KV cache: host bookkeeping of the device table [L][slot][blocks_per_seq] (0 = no page)
+  std::vector<int32_t> bt_host, free_pages;
+  int32_t pages_used;
+  int32_t *bt_dev() const { return reinterpret_cast<int32_t *>(scratch + lay.block_table); }
 
   DevSched *sched() const { return reinterpret_cast<DevSched *>(scratch + lay.sched); }
   float2 *rope() const { return reinterpret_cast<float2 *>(scratch + lay.rope); }
@@ -186,6 +200,40 @@ static const int32_t *thr_for(d3_model *m, double alpha) {
   return it->second.data();
 }
 
+// Paged layout: give every (block, page-sized run of positions) that the rows of this step
+// write a page, before anything is enqueued.  D3_ECAPACITY (nothing changed) when the pool
+// cannot cover the step.  Under D3_FILL_NONE a row takes no page for a block it drops.
+static int32_t pages_for_step(d3_model *m, int B, const int32_t *slot, const int32_t *pos, const int32_t *lo,
+                              const int32_t *hi, int32_t *launches) {
+  const d3_config &c = m->cfg;
+  if (c.kv_layout != D3_KV_PAGED) return D3_OK;
+  const int L = c.n_layers, bps = c.max_seq / c.page_size;
+  auto writes = [&](int b, int l) { return c.kv_fill != D3_FILL_NONE || l < lo[b] || l >= hi[b]; };
+  auto entry = [&](int b, int l) { return ((size_t)l * c.max_slots + slot[b]) * bps + pos[b] / c.page_size; };
+  std::vector<size_t> need;
+  for (int b = 0; b < B; ++b)
+    for (int l = 0; l < L; ++l)
+      if (writes(b, l) && m->bt_host[entry(b, l)] == 0) {
+        size_t e = entry(b, l);
+        bool dup = false;
+        for (size_t q : need) dup = dup || q == e;   // rows of a prefill pass share pages
+        if (!dup) need.push_back(e);
+      }
+  if (need.size() > m->free_pages.size()) return D3_ECAPACITY;
+  TableUpdate u;
+  u.n = 0;
+  for (size_t e : need) {
+    const int32_t page = m->free_pages.back();
+    m->free_pages.pop_back();
+    m->pages_used += 1;
+    m->bt_host[e] = page;
+    u.index[u.n] = (int32_t)e; u.page[u.n] = page;
+    if (++u.n == TableUpdate::kMax) { *launches += launch_table_update(m->bt_dev(), u, m->stream); u.n = 0; }
+  }
+  if (u.n) *launches += launch_table_update(m->bt_dev(), u, m->stream);
+  return D3_OK;
+}
+
 // One projection over `rows` rows: tensor cores for a dense enough group, FMA GEMV otherwise.
 static int project(d3_model *m, const GemvArgs &g, int epi, int rows) {
   const bool tensor = m->exec_mode == D3_EXEC_TENSOR ||
@@ -208,6 +256,10 @@ static int32_t run_step(d3_model *m, const StepArgs &a, const int32_t *n, const 
   cudaStream_t st = m->stream;
   const int B = a.B, L = c.n_layers;
   int launches = 0;
+  {
+    int32_t rc = pages_for_step(m, B, a.slot, a.pos, lo, hi, &launches);
+    if (rc != D3_OK) return rc;
+  }
   { ProfScope ps(m, PK_SCHED); launches += launch_schedule_embed(a, m->sched(), m->embed, m->x(), dm.d, st); }
   const int nq = dm.Hq * dm.dh, nkv = dm.Hkv * dm.dh;
   const int G = dm.Hq / dm.Hkv, GQ = (G % 4 == 0) ? 4 : (G % 2 == 0) ? 2 : 1;
@@ -329,6 +381,23 @@ static int32_t run_fused_step(d3_model *m, const StepArgs &a, float *logits_dev,
   return (rc == 1 && cudaGetLastError() == cudaSuccess) ? D3_OK : D3_ECUDA;
 }
 
+// Paged layout: take back every page of `slot` (host list + device table, in stream order).
+static int32_t release_pages(d3_model *m, int32_t slot) {
+  const d3_config &c = m->cfg;
+  if (c.kv_layout != D3_KV_PAGED) return D3_OK;
+  const int bps = c.max_seq / c.page_size;
+  for (int l = 0; l < c.n_layers; ++l) {
+    int32_t *row = m->bt_host.data() + ((size_t)l * c.max_slots + slot) * bps;
+    bool any = false;
+    for (int k = 0; k < bps; ++k)
+      if (row[k]) { m->free_pages.push_back(row[k]); m->pages_used -= 1; row[k] = 0; any = true; }
+    if (any && cudaMemsetAsync(m->bt_dev() + ((size_t)l * c.max_slots + slot) * bps, 0, bps * sizeof(int32_t),
+                               m->stream) != cudaSuccess)
+      return D3_ECUDA;
+  }
+  return D3_OK;
+}
+
 extern "C" {
 
 int32_t d3_depth(int32_t L, double alpha, int64_t i) {
@@ -377,8 +446,11 @@ int32_t d3_schedule(int32_t L, double alpha, int32_t start_id, int32_t anchor, i
 
 int32_t d3_workspace_bytes(const d3_config *cfg, size_t *kv_bytes, size_t *scratch_bytes) {
   if (!config_ok(cfg) || !kv_bytes || !scratch_bytes) return D3_EINVAL;
-  *kv_bytes = 2 * (size_t)cfg->n_layers * cfg->max_slots * cfg->n_kv_heads * cfg->max_seq *
-              cfg->head_dim * sizeof(bf16);
+  if (cfg->kv_layout == D3_KV_PAGED)
+    *kv_bytes = 2 * (size_t)cfg->n_pages * cfg->n_kv_heads * cfg->page_size * cfg->head_dim * sizeof(bf16);
+  else
+    *kv_bytes = 2 * (size_t)cfg->n_layers * cfg->max_slots * cfg->n_kv_heads * cfg->max_seq *
+                cfg->head_dim * sizeof(bf16);
   *scratch_bytes = make_layout(*cfg).total;
   return D3_OK;
 }
@@ -421,9 +493,29 @@ int32_t d3_load(const d3_config *cfg, const d3_weights *w, void *kv_dev, void *s
     m->w_down.push_back((const bf16 *)w->w_down_dev[l]);
   }
   size_t kv_half = (size_t)L * cfg->max_slots * cfg->n_kv_heads * cfg->max_seq * cfg->head_dim;
+  if (cfg->kv_layout == D3_KV_PAGED)
+    kv_half = (size_t)cfg->n_pages * cfg->n_kv_heads * cfg->page_size * cfg->head_dim;
   m->Kc = (bf16 *)kv_dev;
   m->Vc = m->Kc + kv_half;
   m->scratch = (char *)scratch_dev;
+  m->pages_used = 0;
+  if (cfg->kv_layout == D3_KV_PAGED) {
+    const int ps = cfg->page_size, bps = cfg->max_seq / ps;
+    m->dm.page_size = ps;
+    m->dm.page_shift = 0;
+    while ((1 << m->dm.page_shift) < ps) m->dm.page_shift += 1;
+    m->dm.blocks_per_seq = bps;
+    m->dm.block_table = m->bt_dev();
+    m->bt_host.assign((size_t)L * cfg->max_slots * bps, 0);
+    for (int32_t pg = cfg->n_pages - 1; pg >= 1; --pg) m->free_pages.push_back(pg);   // page 0 reserved
+    const size_t page_bytes = (size_t)cfg->n_kv_heads * ps * cfg->head_dim * sizeof(bf16);
+    if (cudaMemsetAsync(m->bt_dev(), 0, m->bt_host.size() * sizeof(int32_t), m->stream) != cudaSuccess ||
+        cudaMemsetAsync(m->Kc, 0, page_bytes, m->stream) != cudaSuccess ||
+        cudaMemsetAsync(m->Vc, 0, page_bytes, m->stream) != cudaSuccess) {
+      delete m;
+      return D3_ECUDA;
+    }
+  }
   m->pos.assign(cfg->max_slots, -1);
   m->last_B = 0;
   m->prof_on = false;
@@ -472,6 +564,7 @@ int32_t d3_load(const d3_config *cfg, const d3_weights *w, void *kv_dev, void *s
   }
   m->fused_ok = fused_plan(*cfg, &m->fused_grid, &m->fused_stages, &m->fused_act, &m->fused_smem,
                            &m->fused_func);
+  if (cfg->kv_layout != D3_KV_CONTIGUOUS) m->fused_ok = 0;   // the single-kernel step addresses a contiguous cache
   if (m->fused_ok && m->fused_grid > kFusedMaxCtas) m->fused_grid = kFusedMaxCtas;
   if (cudaMemsetAsync(m->sched(), 0, sizeof(DevSched), m->stream) != cudaSuccess ||
       cudaMemsetAsync(m->scratch + m->lay.phase, 0, (size_t)kFusedMaxCtas * kFusedPhases * 8, m->stream) !=
@@ -492,6 +585,8 @@ int32_t d3_prefill(d3_model *m, int32_t slot, const int32_t *tokens, int32_t n_t
   for (int t = 0; t < n_tokens; ++t)
     if (tokens[t] < 0 || tokens[t] >= m->cfg.vocab) return D3_EINVAL;
   const int L = m->cfg.n_layers, MB = m->cfg.max_batch;
+  if (release_pages(m, slot) != D3_OK) return D3_ECUDA;
+  m->pos[slot] = -1;
   const int32_t *thr = thr_for(m, 1.0);
   int32_t n[D3_MAX_BATCH], lo[D3_MAX_BATCH], hi[D3_MAX_BATCH], perm[D3_MAX_BATCH], m_l[D3_MAX_LAYERS];
   for (int t0 = 0; t0 < n_tokens; t0 += MB) {
@@ -610,7 +705,7 @@ int32_t d3_read_kv(d3_model *m, int32_t layer, int32_t slot, int32_t pos, float 
   const int dh = m->cfg.head_dim;
   std::vector<uint16_t> buf(dh);
   for (int h = 0; h < m->cfg.n_kv_heads; ++h) {
-    size_t off = ((((size_t)layer * m->cfg.max_slots + slot) * m->cfg.n_kv_heads + h) * m->cfg.max_seq + pos) * dh;
+    size_t off = kv_offset(m->dm, m->bt_host.data(), layer, slot, h, pos);
     for (int which = 0; which < 2; ++which) {
       const bf16 *src = (which ? m->Vc : m->Kc) + off;
       if (cudaMemcpy(buf.data(), src, dh * 2, cudaMemcpyDeviceToHost) != cudaSuccess) return D3_ECUDA;
@@ -632,7 +727,12 @@ int32_t d3_slot_pos(const d3_model *m, int32_t slot) {
 int32_t d3_reset_slot(d3_model *m, int32_t slot) {
   if (!m || slot < 0 || slot >= m->cfg.max_slots) return D3_EINVAL;
   m->pos[slot] = -1;
-  return D3_OK;
+  return release_pages(m, slot);
+}
+
+int32_t d3_kv_pages_used(const d3_model *m) {
+  if (!m || m->cfg.kv_layout != D3_KV_PAGED) return D3_EINVAL;
+  return m->pages_used;
 }
 
 int32_t d3_sync(d3_model *m) {
@@ -722,7 +822,7 @@ const char *d3_strerror(int32_t code) {
   switch (code) {
     case D3_OK: return "ok";
     case D3_EINVAL: return "invalid argument";
-    case D3_ECAPACITY: return "capacity exceeded (max_seq or max_batch)";
+    case D3_ECAPACITY: return "capacity exceeded (max_seq, max_batch or the page pool)";
     case D3_ESTATE: return "slot not prefilled, or used twice in one batch";
     case D3_ECUDA: return "CUDA runtime error";
     case D3_ETIMEOUT: return "a bounded device-side wait ran out";

@@ -79,7 +79,19 @@ struct GemvArgs {
 
 struct Dims {
   int L, d, Hq, Hkv, dh, f, V, max_slots, max_seq, qkv_rows;
+  // paged KV cache (page_size == 0: contiguous)
+  int page_size, page_shift, blocks_per_seq;
+  const int32_t *block_table;   // device [L][max_slots][blocks_per_seq] page ids; 0 = never written
 };
+
+// Element offset of cache entry (layer, slot, kv head h, position pos) in the K (or V) array.
+__host__ __device__ __forceinline__ size_t kv_offset(const Dims &dm, const int32_t *table, int layer, int slot,
+                                                     int h, int pos) {
+  if (dm.page_size == 0)
+    return ((((size_t)layer * dm.max_slots + slot) * dm.Hkv + h) * dm.max_seq + pos) * (size_t)dm.dh;
+  const int page = table[((size_t)layer * dm.max_slots + slot) * dm.blocks_per_seq + (pos >> dm.page_shift)];
+  return (((size_t)page * dm.Hkv + h) * dm.page_size + (pos & (dm.page_size - 1))) * (size_t)dm.dh;
+}
 
 // device table of one block's weight pointers (fused step kernel)
 struct LayerPtrs {
@@ -126,7 +138,7 @@ struct TcContext {
 // Byte offsets of the regions of the caller's scratch buffer.
 struct Layout {
   size_t sched, rope, x, qkv, attn_out, part_o, part_ml, u, layer_tab, bar, phase, part_fused, act_split,
-      act_split_bytes, total;
+      act_split_bytes, block_table, total;
   int max_splits;
 };
 
@@ -178,6 +190,13 @@ int launch_attention(const float *qkv, const bf16 *Kc, const bf16 *Vc, const Dev
                      float *part_ml, float *attn_out, const Dims &dm, cudaStream_t st);
 int launch_fill_copy(bf16 *Kc, bf16 *Vc, const DevSched *s, int B, const Dims &dm, cudaStream_t st);
 int launch_argmax(const float *logits, int B, int V, int32_t *out, cudaStream_t st);
+// paged KV cache: entries of the device block table that change before a step
+struct TableUpdate {
+  static constexpr int kMax = 256;
+  int32_t n;
+  int32_t index[kMax], page[kMax];
+};
+int launch_table_update(int32_t *table, const TableUpdate &u, cudaStream_t st);
 int init_kernel_attributes();
 // tensor-core projections: 0 when the path is usable on this device / driver
 int tc_init();

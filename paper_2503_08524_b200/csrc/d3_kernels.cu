@@ -354,7 +354,6 @@ k_rope_append(float *qkv, const float2 *rope, bf16 *Kc, bf16 *Vc, const DevSched
   if (hs >= dm.Hq + 2 * dm.Hkv) return;
   const int pos = s->pos_s[row], slot = s->slot_s[row];
   float *p = qkv + (size_t)row * dm.qkv_rows + (size_t)hs * dh;
-  const size_t cbase = ((size_t)layer * dm.max_slots + slot) * dm.Hkv;
   if (hs < dm.Hq) {
     if (kv_only) return;
     const float2 cs = rope[(size_t)pos * half + j];
@@ -364,11 +363,11 @@ k_rope_append(float *qkv, const float2 *rope, bf16 *Kc, bf16 *Vc, const DevSched
   } else if (hs < dm.Hq + dm.Hkv) {
     const float2 cs = rope[(size_t)pos * half + j];
     const float a = p[j], b = p[j + half];
-    bf16 *dst = Kc + ((cbase + (hs - dm.Hq)) * dm.max_seq + pos) * dh;
+    bf16 *dst = Kc + kv_offset(dm, dm.block_table, layer, slot, hs - dm.Hq, pos);
     dst[j] = __float2bfloat16_rn(a * cs.x - b * cs.y);
     dst[j + half] = __float2bfloat16_rn(a * cs.y + b * cs.x);
   } else {
-    bf16 *dst = Vc + ((cbase + (hs - dm.Hq - dm.Hkv)) * dm.max_seq + pos) * dh;
+    bf16 *dst = Vc + kv_offset(dm, dm.block_table, layer, slot, hs - dm.Hq - dm.Hkv, pos);
     dst[j] = __float2bfloat16_rn(p[j]);
     dst[j + half] = __float2bfloat16_rn(p[j + half]);
   }
@@ -428,10 +427,10 @@ k_attn_partial(const float *qkv, const bf16 *Kc, const bf16 *Vc, const DevSched 
 #pragma unroll
     for (int e = 0; e < EPL; ++e) o[g][e] = 0.f;
   }
-  const size_t base = (((size_t)layer * dm.max_slots + slot) * dm.Hkv + kvh) * (size_t)dm.max_seq * DH;
   for (int t = t0 + worker; t < t1; t += 32) {
-    const bf16 *kp = Kc + base + (size_t)t * DH + part * EPL;
-    const bf16 *vp = Vc + base + (size_t)t * DH + part * EPL;
+    const size_t off = kv_offset(dm, dm.block_table, layer, slot, kvh, t) + part * EPL;
+    const bf16 *kp = Kc + off;
+    const bf16 *vp = Vc + off;
     float kf[EPL], vf[EPL];
     if constexpr (EPL == 4) {
       uint2 kw = *reinterpret_cast<const uint2 *>(kp), vw = *reinterpret_cast<const uint2 *>(vp);
@@ -583,12 +582,12 @@ __global__ void k_fill_copy(bf16 *Kc, bf16 *Vc, const DevSched *s, Dims dm) {
   const int n = dm.Hkv * dm.dh;
   for (int i = threadIdx.x; i < n; i += blockDim.x) {
     int h = i / dm.dh, e = i % dm.dh;
-    size_t dst = ((((size_t)l * dm.max_slots + slot) * dm.Hkv + h) * dm.max_seq + pos) * dm.dh + e;
+    size_t dst = kv_offset(dm, dm.block_table, l, slot, h, pos) + e;
     if (lo == 0) {
       Kc[dst] = __float2bfloat16_rn(0.f);
       Vc[dst] = __float2bfloat16_rn(0.f);
     } else {
-      size_t src = ((((size_t)(lo - 1) * dm.max_slots + slot) * dm.Hkv + h) * dm.max_seq + pos) * dm.dh + e;
+      size_t src = kv_offset(dm, dm.block_table, lo - 1, slot, h, pos) + e;
       Kc[dst] = Kc[src];
       Vc[dst] = Vc[src];
     }
@@ -598,6 +597,19 @@ __global__ void k_fill_copy(bf16 *Kc, bf16 *Vc, const DevSched *s, Dims dm) {
 int launch_fill_copy(bf16 *Kc, bf16 *Vc, const DevSched *s, int B, const Dims &dm, cudaStream_t st) {
   dim3 grid(dm.L, B);
   launch_pdl(k_fill_copy, grid, dim3(128), 0, st, Kc, Vc, s, dm);
+  return 1;
+}
+
+// ------------------------------------------------------- paged cache: block table
+__global__ void k_table_update(int32_t *table, const __grid_constant__ TableUpdate u) {
+  pdl_wait();
+  pdl_trigger();
+  const int i = threadIdx.x;
+  if (i < u.n) table[u.index[i]] = u.page[i];
+}
+
+int launch_table_update(int32_t *table, const TableUpdate &u, cudaStream_t st) {
+  launch_pdl(k_table_update, dim3(1), dim3(TableUpdate::kMax), 0, st, table, u);
   return 1;
 }
 

@@ -44,6 +44,7 @@ extern "C" int32_t d3_decode_step_noalloc(const d3_config *cfg, const d3_weights
                                           int32_t slot, int32_t pos, int32_t token, int32_t gen_index,
                                           double alpha, float *logits_dev, void *cuda_stream) {
   if (!config_ok(cfg) || !w || !kv_dev || !logits_dev) return D3_EINVAL;
+  if (cfg->kv_layout != D3_KV_CONTIGUOUS) return D3_EINVAL;   // the page table lives in a model handle
   if (!w->embed_dev || !w->lm_head_dev || !w->final_norm_dev || !w->attn_norm_dev || !w->wqkv_dev ||
       !w->wo_dev || !w->mlp_norm_dev || !w->w_gate_dev || !w->w_up_dev || !w->w_down_dev)
     return D3_EINVAL;

@@ -20,7 +20,7 @@ def rel_l2(a, b):
 
 
 def make_pair(shape, seed, max_slots, max_seq, max_batch, start_id=0, anchor=0, kv_fill=1,
-              gain_jitter=0.1, gen_device="cuda:0", kv_round_bf16=True):
+              gain_jitter=0.1, gen_device="cuda:0", kv_round_bf16=True, page_size=0, n_pages=0):
     """(oracle, gpu model) over identical weights.  Weights are generated once
     (integer hash, bit-identical on either device) and copied to the other side.
     kv_round_bf16: the oracle stores K and V rounded to bf16, the cache format
@@ -33,7 +33,7 @@ def make_pair(shape, seed, max_slots, max_seq, max_batch, start_id=0, anchor=0, 
     orc = O.Oracle(shape, w_cpu, max_slots, max_seq, start_id=start_id, anchor=anchor, kv_fill=kv_fill,
                    kv_round_bf16=kv_round_bf16)
     gpu = B.D3Model(shape, w_dev, max_slots, max_seq, max_batch, start_id=start_id, anchor=anchor,
-                    kv_fill=kv_fill)
+                    kv_fill=kv_fill, page_size=page_size, n_pages=n_pages)
     return orc, gpu
 
 

@@ -126,13 +126,15 @@ def test_tiny_greedy_tokens_identical(B):
 
 @pytest.mark.parametrize("anchor,start", [(0, 0), (0, 1), (0, 2), (1, 0)])
 @pytest.mark.parametrize("fill", [0, 1, 2])
-@pytest.mark.parametrize("exec_mode", [0, 1], ids=["tensor-cores", "fma"])
-def test_batched_mixed_depth_steps(B, anchor, start, fill, exec_mode):
+@pytest.mark.parametrize("exec_mode,paged", [(0, False), (1, False), (0, True)],
+                         ids=["tensor-cores", "fma", "paged-kv"])
+def test_batched_mixed_depth_steps(B, anchor, start, fill, exec_mode, paged):
     # exec 0: depth groups of 2+ rows project on the tensor cores, single rows by FMA GEMV;
-    # exec 1: FMA GEMVs throughout
+    # exec 1: FMA GEMVs throughout; paged: the cache is a pool of 16-position pages
     shape = I.TINY_GQA
     Bn, alpha = 7, 0.96
-    orc, gpu = make_pair(shape, SEED + 2, 8, 96, 8, start_id=start, anchor=anchor, kv_fill=fill)
+    pk = dict(page_size=16, n_pages=1 + shape.n_layers * 8 * 6) if paged else {}
+    orc, gpu = make_pair(shape, SEED + 2, 8, 96, 8, start_id=start, anchor=anchor, kv_fill=fill, **pk)
     gpu.d3_set_exec(exec_mode)
     gpu.poison_kv()
     orc.poison_kv()
@@ -242,14 +244,19 @@ def test_prefill_longer_than_a_batch_and_ragged_lengths(B):
 
 @pytest.mark.parametrize("base,layers,Bn", [(I.LLAMA_7B, 3, 1), (I.LLAMA_7B, 2, 5), (I.LLAMA_70B, 2, 3),
                                             (I.LLAMA_13B, 2, 1), (I.LLAMA_70B, 2, 1), (I.LLAMA_7B, 2, 32),
-                                            (I.LLAMA_13B, 2, 8), (I.LLAMA_70B, 2, 4)],
+                                            (I.LLAMA_13B, 2, 8), (I.LLAMA_70B, 2, 4), (I.LLAMA_7B, 2, -5)],
                          ids=["7b-width-b1", "7b-width-b5", "70b-width-gqa-b3", "13b-width-b1",
-                              "70b-width-gqa-b1", "7b-width-b32", "13b-width-b8", "70b-width-gqa-b4"])
+                              "70b-width-gqa-b1", "7b-width-b32", "13b-width-b8", "70b-width-gqa-b4",
+                              "7b-width-b5-paged-kv"])
 def test_production_widths(B, base, layers, Bn):
     # full-width blocks (same kernel shapes and tiling as the benchmark), few layers;
     # batches of 2+ rows take the tensor-core projections, single rows the fused step
     shape = base.with_layers(layers)
-    orc, gpu = make_pair(shape, SEED + 5, Bn, 96, max(8, Bn), start_id=1, gain_jitter=0.1)
+    pk = {}
+    if Bn < 0:      # negative row count: the same case over a paged cache (32-position pages)
+        Bn = -Bn
+        pk = dict(page_size=32, n_pages=1 + layers * Bn * 3)
+    orc, gpu = make_pair(shape, SEED + 5, Bn, 96, max(8, Bn), start_id=1, gain_jitter=0.1, **pk)
     lens = I.uniform_ints(SEED + 5, 3, Bn, 5, 40 if Bn <= 8 else 12)
     for b in range(Bn):
         p = I.prompt_tokens(shape, SEED + 5, b, lens[b]).numpy()
@@ -264,6 +271,70 @@ def test_production_widths(B, base, layers, Bn):
         g = gpu.d3_decode_step(list(range(Bn)), toks, gi, alpha)
         check_step(f"step {step}", g.cpu().numpy(), gpu.d3_read_hidden(Bn), r["logits"], r["hidden"])
     gpu.d3_sync()          # raises on a deferred device status (a bounded wait that ran out)
+    gpu.close()
+
+
+# ------------------------------------------------------------------ paged KV cache
+
+def test_paged_cache_single_row_run_and_page_accounting(B):
+    # batch 1 over a paged cache (sequence of kernels), depth decaying over page boundaries.
+    # FILL_NONE never writes a dropped (token, block) pair, so a block stops taking pages once
+    # the tokens stop running it; FILL_COPY writes every pair and takes pages like a dense cache.
+    shape = I.TINY
+    L, ps, alpha, start = shape.n_layers, 16, 0.93, 1
+    used = {}
+    for fill in (0, 1):
+        orc, gpu = make_pair(shape, SEED + 9, 2, 96, 4, start_id=start, kv_fill=fill, page_size=ps,
+                             n_pages=1 + 2 * L * 6)
+        gpu.poison_kv()
+        orc.poison_kv()
+        prompt = I.prompt_tokens(shape, SEED + 9, 0, 21).numpy()
+        o = orc.prefill(0, prompt)
+        g = gpu.d3_prefill(0, prompt)
+        check_step("prefill", g.cpu().numpy()[None], None, o[None], None)
+        assert gpu.d3_kv_pages_used() == L * 2                      # positions 0..20: two pages per block
+        written = {(l, p // ps) for l in range(L) for p in range(21)}
+        toks = I.token_ids(SEED + 9, 5, 64, shape.vocab).numpy()
+        for i in range(1, 50):
+            pos = orc.slot_pos(0)
+            r = orc.decode_step([0], [int(toks[i])], [i], alpha)
+            g = gpu.d3_decode_step([0], [int(toks[i])], [i], alpha)
+            check_step(f"step {i}", g.cpu().numpy(), gpu.d3_read_hidden(1), r["logits"], r["hidden"])
+            n, lo, hi = O.window(L, alpha, i, start)
+            for l in range(L):
+                if fill != 0 or not (lo <= l < hi):
+                    written.add((l, pos // ps))
+            assert gpu.d3_kv_pages_used() == len(written), (fill, i)
+        used[fill] = gpu.d3_kv_pages_used()
+        # a second sequence takes its own pages; resetting it gives exactly those back
+        gpu.d3_prefill(1, prompt[:5])
+        assert gpu.d3_kv_pages_used() == used[fill] + L
+        gpu.d3_reset_slot(1)
+        assert gpu.d3_kv_pages_used() == used[fill]
+        gpu.d3_sync()
+        gpu.close()
+    assert used[1] == L * 5                                          # 70 positions, dense
+    assert used[0] < used[1]                                         # the depth-aware saving
+
+
+def test_paged_pool_exhaustion_is_an_error_and_changes_nothing(B):
+    shape = I.TINY
+    L = shape.n_layers
+    orc, gpu = make_pair(shape, SEED + 10, 2, 64, 4, page_size=16, n_pages=1 + 2 * L)
+    p = I.prompt_tokens(shape, SEED + 10, 0, 16).numpy()
+    gpu.d3_prefill(0, p)                       # L pages
+    gpu.d3_prefill(1, p[:3])                   # L pages: the pool is now empty
+    orc.prefill(0, p)
+    assert gpu.d3_kv_pages_used() == 2 * L
+    with pytest.raises(B.D3Error) as e:     # position 16 of slot 0 needs a new page per block
+        gpu.d3_decode_step([0], [5], [1], 1.0)
+    assert e.value.code == B.ECAPACITY
+    assert gpu.d3_slot_pos(0) == 16 and gpu.d3_kv_pages_used() == 2 * L
+    gpu.d3_reset_slot(1)                       # pages come back; the step now goes through
+    r = orc.decode_step([0], [5], [1], 1.0)
+    g = gpu.d3_decode_step([0], [5], [1], 1.0)
+    check_step("after reset", g.cpu().numpy(), gpu.d3_read_hidden(1), r["logits"], r["hidden"])
+    gpu.d3_sync()
     gpu.close()
 
 

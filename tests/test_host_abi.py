@@ -95,6 +95,18 @@ def test_workspace_and_load_validation():
         with pytest.raises(B.D3Error) as e:
             B.d3_workspace_bytes(c)
         assert e.value.code == B.EINVAL, field
+    # paged layout: pool of n_pages pages of page_size positions, one block each
+    pc = B.make_config(I.LLAMA_7B, 4, 1024, 4, page_size=64, n_pages=100)
+    pkv, pscratch = B.d3_workspace_bytes(pc)
+    assert pkv == 2 * 100 * 32 * 64 * 128 * 2
+    assert pscratch > B.d3_workspace_bytes(B.make_config(I.LLAMA_7B, 4, 1024, 4))[1]   # + the page table
+    for field, bad in [("page_size", 48), ("page_size", 8), ("page_size", 2048), ("n_pages", 1),
+                       ("max_seq", 1000), ("kv_layout", 0)]:
+        c = B.make_config(I.LLAMA_7B, 4, 1024, 4, page_size=64, n_pages=100)
+        setattr(c, field, bad)
+        with pytest.raises(B.D3Error) as e:
+            B.d3_workspace_bytes(c)
+        assert e.value.code == B.EINVAL, field
     h = C.c_void_p()
     assert B.LIB.d3_load(C.byref(cfg), None, None, None, None, C.byref(h)) == B.EINVAL
     assert B.LIB.d3_load(None, None, None, None, None, C.byref(h)) == B.EINVAL
