@@ -183,7 +183,7 @@ int32_t d3_read_kv(d3_model *m, int32_t layer, int32_t slot, int32_t pos, float 
 /* How decode steps execute.  AUTO: a batch of one row runs as a single persistent
  * cooperative kernel when the device and sizes allow it (fill modes NONE and
  * COPY), everything else as a sequence of kernels per block, whose projections
- * run on the tensor cores (tcgen05, bf16 hi+lo split activations, fp32
+ * run on the tensor cores (tcgen05, activations split exactly into three bf16 terms, fp32
  * accumulate) once the block's depth group has D3_TENSOR_MIN_ROWS rows or more and
  * as FP32-FMA GEMVs below that.  KERNELS: always the sequence of kernels with
  * FMA GEMVs.  TENSOR: always the sequence of kernels with tensor-core

@@ -21,6 +21,7 @@ FILL_NONE, FILL_COPY, FILL_RECOMPUTE = 0, 1, 2
 MAX_BATCH, MAX_LAYERS, PROF_KINDS = 64, 128, 22
 EXEC_AUTO, EXEC_KERNELS, EXEC_TENSOR = 0, 1, 2
 KV_CONTIGUOUS, KV_PAGED = 0, 1
+MAX_BATCH = 64     # D3_MAX_BATCH
 
 EXPORTS = ("d3_depth", "d3_schedule", "d3_workspace_bytes", "d3_load", "d3_prefill",
            "d3_decode_step", "d3_argmax", "d3_read_schedule", "d3_read_hidden", "d3_read_kv",
@@ -272,11 +273,14 @@ class D3Model:
                 "rows_layers": int(cnt[0]), "layers_touched": int(cnt[1])}
 
     def d3_read_hidden(self, B: int) -> np.ndarray:
-        out = np.zeros((B, self.shape.d_model), np.float32)
+        """Residual stream of the last step's rows (caller order).  The library writes as many
+        rows as that step had (a prefill pass: up to max_batch), so the buffer is sized for the
+        largest step; the first B rows are returned, or the LAST row when B == -1."""
+        out = np.zeros((MAX_BATCH, self.shape.d_model), np.float32)
         rc = LIB.d3_read_hidden(self.h, out.ctypes.data)
         if rc != OK:
             raise D3Error(rc, "d3_read_hidden")
-        return out
+        return out[:B].copy()
 
     def d3_read_kv(self, layer: int, slot: int, pos: int):
         n = self.shape.n_kv_heads * self.shape.head_dim

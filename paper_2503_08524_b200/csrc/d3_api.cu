@@ -32,12 +32,12 @@ Layout make_layout(const d3_config &c) {
   y.phase = off;    off = align_up(off + (size_t)kFusedMaxCtas * kFusedPhases * 8, 256);
   y.part_fused = off;
   off = align_up(off + (size_t)c.n_q_heads * kFusedMaxCtas * (c.head_dim + 2) * 4, 256);
-  // tensor-core operand: bf16 hi rows + lo rows of the widest activation
+  // tensor-core operand: bf16 hi, mid and lo rows of the widest activation
   size_t kmax = (size_t)c.d_model;
   if ((size_t)c.n_q_heads * c.head_dim > kmax) kmax = (size_t)c.n_q_heads * c.head_dim;
   if ((size_t)c.d_ffn > kmax) kmax = (size_t)c.d_ffn;
   y.act_split = off = align_up(off, 1024);
-  y.act_split_bytes = 2 * ((B + 7) / 8 * 8) * kmax * sizeof(bf16);
+  y.act_split_bytes = 3 * ((B + 15) / 16 * 16) * kmax * sizeof(bf16);
   off = align_up(off + y.act_split_bytes, 256);
   y.block_table = off;
   if (c.kv_layout == D3_KV_PAGED)

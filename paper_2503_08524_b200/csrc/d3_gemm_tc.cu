@@ -8,12 +8,14 @@
 //
 // Operand roles are swapped with respect to the usual GEMM: the WEIGHT tile is
 // the 128-row "A" operand (UMMA M = 128), the activations are the narrow "B"
-// operand (UMMA N = 2 * padded rows).  The fp32 activations are split by a
+// operand (UMMA N = 3 * padded rows).  The fp32 activations are split by a
 // small pre-pass (k_act_split, which also applies the fused RMSNorm) into
-// bf16 hi + bf16 lo with hi + lo = act to 2^-17 relative: both halves sit side by side in N,
-// and the epilogue adds the two accumulator columns of a row.  The products are
-// exact in the fp32 accumulator, so the result differs from the fp32-activation
-// FMA path only by the 2^-17 split error and the summation order.
+// three bf16 terms hi + mid + lo = act exactly (3 x 8 significand bits cover
+// fp32's 24): the three sit side by side in N and the epilogue adds the three
+// accumulator columns of a row.  The products are exact in the fp32
+// accumulator, so the result differs from the fp32-activation FMA path only by
+// the summation order.  (Two terms leave a 2^-17 relative error; at 32 blocks
+// that flips enough bf16 roundings of cached K and V to double the logit error.)
 //
 // One CTA = one tile of 128 weight rows (two 64-row TMA boxes: rows r..r+63 and
 // r+64..r+127 of one matrix, or 64 gate rows + the same 64 up rows for SwiGLU)
@@ -73,7 +75,7 @@ __device__ __forceinline__ uint32_t bar_try_wait(uint32_t bar, uint32_t parity) 
 
 struct TcArgs {
   int R, K;              // weight rows (outputs), reduction length
-  int NP;                // padded activation rows, a multiple of 8; UMMA N = 2 NP
+  int NP;                // padded activation rows, a multiple of 16; UMMA N = 3 NP
   int n_kb, kb_per_split;
   int n_stages, tmem_cols;
   int atomic;            // combine with red.add (split-K or residual)
@@ -150,6 +152,15 @@ __device__ __forceinline__ void tmem_ld8(uint32_t taddr, float (&v)[8]) {
 #pragma unroll
   for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(r[i]);
 }
+// y[i] = the three accumulator columns (hi, mid, lo term) of activation rows j0 .. j0+7, small first
+__device__ __forceinline__ void tmem_sum3(uint32_t tbase, int j0, int NP, float (&y)[8]) {
+  float hi[8], mid[8], lo[8];
+  tmem_ld8(tbase + (uint32_t)j0, hi);
+  tmem_ld8(tbase + (uint32_t)(NP + j0), mid);
+  tmem_ld8(tbase + (uint32_t)(2 * NP + j0), lo);
+#pragma unroll
+  for (int i = 0; i < 8; ++i) y[i] = (lo[i] + mid[i]) + hi[i];
+}
 __device__ __forceinline__ void fence_before_sync() {
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
 }
@@ -185,7 +196,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
   }
   const int n_it = kb1 - kb0;
   const int S = t.n_stages;
-  const int N = 2 * t.NP;
+  const int N = 3 * t.NP;
   const uint32_t stage_bytes = (uint32_t)(kABytes + N * kTileK * 2);
   // the swizzle pattern is a function of the address: tiles start on 1024-byte boundaries
   const uint32_t ring = (smem_addr(tc_smem_raw) + 1023u) & ~1023u;
@@ -294,25 +305,23 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
     if (EPI == EPI_SWIGLU) {
       if (live && trow >= kBoxRows) {
         for (int j0 = 0; j0 < nrows; j0 += 8) {
-          float hi[8], lo[8];
-          tmem_ld8(tbase + (uint32_t)j0, hi);
-          tmem_ld8(tbase + (uint32_t)(t.NP + j0), lo);
+          float y[8];
+          tmem_sum3(tbase, j0, t.NP, y);
 #pragma unroll
-          for (int i = 0; i < 8; ++i) xch[(j0 + i) * kBoxRows + (trow - kBoxRows)] = hi[i] + lo[i];
+          for (int i = 0; i < 8; ++i) xch[(j0 + i) * kBoxRows + (trow - kBoxRows)] = y[i];
         }
       }
       epilogue_sync();
       const int r = blockIdx.x * kBoxRows + trow;
       if (live && trow < kBoxRows) {
         for (int j0 = 0; j0 < nrows; j0 += 8) {
-          float hi[8], lo[8];
-          tmem_ld8(tbase + (uint32_t)j0, hi);
-          tmem_ld8(tbase + (uint32_t)(t.NP + j0), lo);
+          float y[8];
+          tmem_sum3(tbase, j0, t.NP, y);
 #pragma unroll
           for (int i = 0; i < 8; ++i) {
             const int j = j0 + i;
             if (j < nrows && r < t.R) {
-              const float z = hi[i] + lo[i], up = xch[j * kBoxRows + trow];
+              const float z = y[i], up = xch[j * kBoxRows + trow];
               t.out[(size_t)(r0 + j) * t.out_stride + t.out_col0 + r] = z / (1.f + __expf(-z)) * up;
             }
           }
@@ -321,9 +330,8 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
     } else if (live) {
       const int r = blockIdx.x * kTileM + trow;
       for (int j0 = 0; j0 < nrows; j0 += 8) {
-        float hi[8], lo[8];
-        tmem_ld8(tbase + (uint32_t)j0, hi);
-        tmem_ld8(tbase + (uint32_t)(t.NP + j0), lo);
+        float y[8];
+        tmem_sum3(tbase, j0, t.NP, y);
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
           const int j = j0 + i;
@@ -331,9 +339,8 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
             const int row = r0 + j;
             const int orow = (EPI == EPI_LOGITS) ? (t.row_mode == ROWS_LAST ? 0 : t.sched->perm[row]) : row;
             float *o = t.out + (size_t)orow * t.out_stride + t.out_col0 + r;
-            const float y = hi[i] + lo[i];
-            if (t.atomic) asm volatile("red.global.add.f32 [%0], %1;" ::"l"(o), "f"(y) : "memory");
-            else *o = y;
+            if (t.atomic) asm volatile("red.global.add.f32 [%0], %1;" ::"l"(o), "f"(y[i]) : "memory");
+            else *o = y[i];
           }
         }
       }
@@ -350,8 +357,8 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
 }
 
 // -------------------------------------------------------------- the pre-pass
-// Row j of the group: act' = act (or RMSNorm(act) * gain), written as bf16 hi
-// in row j and bf16 lo in row NP + j of the operand buffer.  When the GEMM
+// Row j of the group: act' = act (or RMSNorm(act) * gain), written as three bf16
+// terms in rows j, NP + j and 2 NP + j of the operand buffer (hi + mid + lo = act').  When the GEMM
 // combines split-K slices into a plain (non-residual) output, the pre-pass also
 // zeroes that output row.
 struct SplitArgs {
@@ -359,7 +366,7 @@ struct SplitArgs {
   int act_stride, K, NP;
   const bf16 *gain;
   float eps;
-  bf16 *dst;             // [2 NP][K]
+  bf16 *dst;             // [3 NP][K]
   float *zero_out;       // nullable
   int out_stride, out_col0, R;
   const DevSched *sched;
@@ -398,7 +405,8 @@ __global__ void __launch_bounds__(256) k_act_split(const SplitArgs a) {
     __syncthreads();
     sc = s_scale;
   }
-  bf16 *hi = a.dst + (size_t)j * a.K, *lo = a.dst + (size_t)(a.NP + j) * a.K;
+  bf16 *hi = a.dst + (size_t)j * a.K, *mid = a.dst + (size_t)(a.NP + j) * a.K,
+       *lo = a.dst + (size_t)(2 * a.NP + j) * a.K;
   const int k = blockIdx.y * 1024 + tid * 4;
   if (k < a.K) {
     float4 v = *reinterpret_cast<const float4 *>(src + k);
@@ -408,13 +416,16 @@ __global__ void __launch_bounds__(256) k_act_split(const SplitArgs a) {
       v.z *= sc * __uint_as_float(gw.y << 16); v.w *= sc * __uint_as_float(gw.y & 0xffff0000u);
     }
     const float f[4] = {v.x, v.y, v.z, v.w};
-    __align__(8) bf16 h[4], l[4];
+    __align__(8) bf16 h[4], md[4], l[4];
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
       h[i] = __float2bfloat16_rn(f[i]);
-      l[i] = __float2bfloat16_rn(f[i] - __bfloat162float(h[i]));
+      const float r1 = f[i] - __bfloat162float(h[i]);     // exact
+      md[i] = __float2bfloat16_rn(r1);
+      l[i] = __float2bfloat16_rn(r1 - __bfloat162float(md[i]));
     }
     *reinterpret_cast<uint2 *>(hi + k) = *reinterpret_cast<const uint2 *>(h);
+    *reinterpret_cast<uint2 *>(mid + k) = *reinterpret_cast<const uint2 *>(md);
     *reinterpret_cast<uint2 *>(lo + k) = *reinterpret_cast<const uint2 *>(l);
   }
   if (a.zero_out) {
@@ -482,7 +493,7 @@ int tc_init() {
 int launch_gemm_tc(TcContext &tc, const GemvArgs &g, int epi, int m_rows, cudaStream_t st) {
   if (!tc.ok || !g.tmap_w || m_rows < 1 || m_rows > D3_MAX_BATCH) return 0;
   if (epi == EPI_SWIGLU && !g.tmap_w2) return 0;
-  const int NP = (m_rows + 7) / 8 * 8, N = 2 * NP;
+  const int NP = (m_rows + 15) / 16 * 16, N = 3 * NP;   // N is a multiple of 16 (UMMA M = 128), <= 192
   if ((size_t)N * g.K * sizeof(bf16) > tc.act_bytes) return 0;
   const uint64_t key = ((uint64_t)NP << 32) | (uint32_t)g.K;
   auto it = tc.act_maps.find(key);

@@ -128,7 +128,7 @@ struct FusedParams {
 // Host state of the tensor-core projection path.
 struct TcContext {
   bool ok;                              // the driver's tensor-map encoder is there and the kernels are set up
-  bf16 *act_split;                      // device: activations as bf16 hi rows then lo rows, [2 NP][K]
+  bf16 *act_split;                      // device: activations as bf16 hi, mid, lo rows, [3 NP][K]
   size_t act_bytes;
   std::map<uint64_t, TMap> act_maps;    // tensor maps of act_split, keyed by (NP, K)
   int sm_count;
