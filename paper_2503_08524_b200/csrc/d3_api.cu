@@ -37,7 +37,7 @@ Layout make_layout(const d3_config &c) {
   if ((size_t)c.n_q_heads * c.head_dim > kmax) kmax = (size_t)c.n_q_heads * c.head_dim;
   if ((size_t)c.d_ffn > kmax) kmax = (size_t)c.d_ffn;
   y.act_split = off = align_up(off, 1024);
-  y.act_split_bytes = 3 * ((B + 15) / 16 * 16) * kmax * sizeof(bf16);
+  y.act_split_bytes = (3 * ((B + 7) / 8 * 8) + 8) * kmax * sizeof(bf16);
   off = align_up(off + y.act_split_bytes, 256);
   y.block_table = off;
   if (c.kv_layout == D3_KV_PAGED)

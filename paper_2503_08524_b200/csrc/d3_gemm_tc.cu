@@ -75,7 +75,8 @@ __device__ __forceinline__ uint32_t bar_try_wait(uint32_t bar, uint32_t parity) 
 
 struct TcArgs {
   int R, K;              // weight rows (outputs), reduction length
-  int NP;                // padded activation rows, a multiple of 16; UMMA N = 3 NP
+  int NP;                // padded activation rows, a multiple of 8
+  int N;                 // UMMA N = 3 NP rounded up to a multiple of 16 (the spare columns are not read)
   int n_kb, kb_per_split;
   int n_stages, tmem_cols;
   int atomic;            // combine with red.add (split-K or residual)
@@ -196,7 +197,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
   }
   const int n_it = kb1 - kb0;
   const int S = t.n_stages;
-  const int N = 3 * t.NP;
+  const int N = t.N;
   const uint32_t stage_bytes = (uint32_t)(kABytes + N * kTileK * 2);
   // the swizzle pattern is a function of the address: tiles start on 1024-byte boundaries
   const uint32_t ring = (smem_addr(tc_smem_raw) + 1023u) & ~1023u;
@@ -493,7 +494,9 @@ int tc_init() {
 int launch_gemm_tc(TcContext &tc, const GemvArgs &g, int epi, int m_rows, cudaStream_t st) {
   if (!tc.ok || !g.tmap_w || m_rows < 1 || m_rows > D3_MAX_BATCH) return 0;
   if (epi == EPI_SWIGLU && !g.tmap_w2) return 0;
-  const int NP = (m_rows + 15) / 16 * 16, N = 3 * NP;   // N is a multiple of 16 (UMMA M = 128), <= 192
+  // three operand rows per activation row; UMMA M = 128 wants N a multiple of 16 (<= 192 here):
+  // up to 8 spare rows of the operand buffer ride along (whatever they hold, their columns are unused)
+  const int NP = (m_rows + 7) / 8 * 8, N = (3 * NP + 15) / 16 * 16;
   if ((size_t)N * g.K * sizeof(bf16) > tc.act_bytes) return 0;
   const uint64_t key = ((uint64_t)NP << 32) | (uint32_t)g.K;
   auto it = tc.act_maps.find(key);
@@ -526,10 +529,13 @@ int launch_gemm_tc(TcContext &tc, const GemvArgs &g, int epi, int m_rows, cudaSt
   launch_pdl(k_act_split, dim3(m_rows, (g.K + 1023) / 1024), dim3(256), 0, st, sa);
 
   TcArgs t;
-  t.R = g.R; t.K = g.K; t.NP = NP; t.n_kb = n_kb; t.kb_per_split = per;
+  t.R = g.R; t.K = g.K; t.NP = NP; t.N = N; t.n_kb = n_kb; t.kb_per_split = per;
   const int stage_bytes = kABytes + N * kTileK * 2;
   t.n_stages = kSmemBudget / stage_bytes;
   if (t.n_stages > kMaxStagesTc) t.n_stages = kMaxStagesTc;
+  // Measured: a fifth stage does not shorten any launch, but its shared memory keeps the next
+  // kernel's CTAs from becoming resident early (13B shape, 8 rows: 7.24 ms per step with 5, 6.43 with 4).
+  if (t.n_stages > 4) t.n_stages = 4;
   if (t.n_stages > per) t.n_stages = per < 2 ? 2 : per;
   t.tmem_cols = 32;
   while (t.tmem_cols < N) t.tmem_cols *= 2;
