@@ -76,6 +76,11 @@ def _lib(kind: str) -> C.CDLL:
                                     C.c_void_p]
         lib.d3o_decode_step.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p,
                                         C.c_double, C.c_void_p, C.c_void_p, C.c_void_p]
+        lib.d3o_decode_step_depths.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p,
+                                               C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+        lib.d3o_depth_linear.argtypes = [C.c_int32, C.c_int32, C.c_int64, C.c_int64]
+        lib.d3o_window_of_depth.argtypes = [C.c_int32, C.c_int32, C.c_int32, C.c_int32,
+                                            C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
         lib.d3o_decode_layers.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_int32,
                                           C.c_void_p, C.c_void_p]
         lib.d3o_forward_nocache.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p]
@@ -98,6 +103,18 @@ def depth(L: int, alpha: float, i: int) -> int:
 
 def depth_pow(L: int, alpha: float, i: int) -> int:
     return int(_lib("f64").d3o_depth_pow(L, alpha, i))
+
+
+def depth_linear(upper: int, lower: int, span: int, i: int) -> int:
+    """Linear decay from `upper` layers at i = 0 to `lower` at i = span, constant after."""
+    return int(_lib("f64").d3o_depth_linear(upper, lower, span, i))
+
+
+def window_of_depth(L: int, n: int, start_id: int, anchor: int = ANCHOR_START):
+    """(retained count, lo, hi) for a retained count given by the caller."""
+    lo, hi = C.c_int32(), C.c_int32()
+    r = _lib("f64").d3o_window_of_depth(L, n, start_id, anchor, C.byref(lo), C.byref(hi))
+    return int(r), int(lo.value), int(hi.value)
 
 
 def window(L: int, alpha: float, i: int, start_id: int, anchor: int = ANCHOR_START):
@@ -215,6 +232,20 @@ class Oracle:
         if want_trace:
             out["trace"] = trace
         return out
+
+    def decode_step_depths(self, slots, tokens, depths):
+        """One generation step with the retained count of every row given by the caller."""
+        B = len(slots)
+        s = np.ascontiguousarray(np.asarray(slots, dtype=np.int32))
+        t = np.ascontiguousarray(np.asarray(tokens, dtype=np.int32))
+        n = np.ascontiguousarray(np.asarray(depths, dtype=np.int32))
+        logits = np.zeros((B, self.shape.vocab), np.float64)
+        hidden = np.zeros((B, self.shape.d_model), np.float64)
+        rc = self.lib.d3o_decode_step_depths(self.h, B, s.ctypes.data, t.ctypes.data, n.ctypes.data,
+                                             logits.ctypes.data, hidden.ctypes.data, None)
+        if rc != 0:
+            raise ValueError(f"oracle decode_step_depths failed ({rc})")
+        return {"logits": logits, "hidden": hidden}
 
     def decode_layers(self, slot: int, token: int, layers: Sequence[int]):
         """One step over exactly the listed blocks (no schedule, no fill)."""

@@ -31,6 +31,10 @@
  *   fill modes          logits independent of the fill mode under a fixed
  *                       (alpha, start), skipped entries poisoned with NaN
  *   textbook properties softmax, RMSNorm, RoPE closed forms and invariants
+ *   caller-given depths the step with depths = floor(L alpha^i) equals the alpha step
+ *                       (itself pinned above); linear decay: end points, monotonicity
+ *                       and the floor-sum identity sum_{i<n} floor(a i / n) =
+ *                       ((a-1)(n-1) + gcd(a,n) - 1) / 2
  * Parity unpinned: the VALUES that fill modes COPY / RECOMPUTE leave in the
  * cache when the caller raises alpha between steps (the paper never states
  * which rule D3 itself uses); only their own definitions below fix them.
@@ -187,9 +191,37 @@ int32_t d3o_depth_pow(int32_t L, double alpha, int64_t i) {
  * at start_id and holds L - n layers, n never falling below start_id so that
  * the window ends at the last layer at the latest.
  * TAIL (the Early-Exit direction, Sec. 1 (ii)): the last L - n layers. */
+static int32_t window_of_depth(int32_t L, int32_t n, int32_t start_id, int32_t anchor, int32_t *lo,
+                               int32_t *hi);
+
 int32_t d3o_window(int32_t L, double alpha, int64_t i, int32_t start_id, int32_t anchor,
                    int32_t *lo, int32_t *hi) {
-  int32_t n = d3o_depth(L, alpha, i);
+  return window_of_depth(L, d3o_depth(L, alpha, i), start_id, anchor, lo, hi);
+}
+
+/* The same window for a retained count n given by the caller (any schedule). */
+int32_t d3o_window_of_depth(int32_t L, int32_t n, int32_t start_id, int32_t anchor, int32_t *lo,
+                            int32_t *hi) {
+  if (n > L) return -1;
+  return window_of_depth(L, n, start_id, anchor, lo, hi);
+}
+
+/* Linear decay between an upper and a lower bound of executed layers (the shape
+ * the paper ascribes to SkipDecode, Sec. 3.4 and Sec. 4.1 "Comparison Methods";
+ * its constants are not given there, so they are parameters): the count falls
+ * from `upper` at i = 0 to `lower` at i = span in equal steps and stays there,
+ *   n(i) = upper - floor((upper - lower) * min(i, span) / span). */
+int32_t d3o_depth_linear(int32_t upper, int32_t lower, int64_t span, int64_t i) {
+  if (upper < 0 || lower < 0 || lower > upper || span < 1 || i < 0) return -1;
+  int64_t t = i < span ? i : span;
+  int64_t drop = 0; /* floor(D * t / span) by counting: D * t = drop * span + rest */
+  int64_t num = (int64_t)(upper - lower) * t;
+  while ((drop + 1) * span <= num) ++drop;
+  return (int32_t)(upper - drop);
+}
+
+static int32_t window_of_depth(int32_t L, int32_t n, int32_t start_id, int32_t anchor, int32_t *lo,
+                               int32_t *hi) {
   if (n < 0 || start_id < 0 || start_id > L) return -1;
   if (anchor == D3O_ANCHOR_TAIL) {
     *lo = n;
@@ -472,15 +504,44 @@ int32_t d3o_prefill(d3o_model *m, int32_t slot, const int32_t *tokens, int32_t n
  *   logits  [B][vocab]; hidden (nullable) [B][d] residual stream before the
  *   final norm; trace (nullable) [B][L+1][d] residual stream before block 0
  *   and after every layer. */
+static int32_t step_with_depths(d3o_model *m, int32_t B, const int32_t *slots, const int32_t *tokens,
+                                const int32_t *depths, double *logits, double *hidden,
+                                double *trace);
+
 int32_t d3o_decode_step(d3o_model *m, int32_t B, const int32_t *slots, const int32_t *tokens,
                         const int32_t *gen_index, double alpha, double *logits,
                         double *hidden, double *trace) {
+  if (B < 1 || !(alpha > 0.0) || !(alpha <= 1.0)) return -1;
+  int32_t *depths = (int32_t *)malloc(sizeof(int32_t) * (size_t)B);
+  for (int b = 0; b < B; ++b) {
+    if (gen_index[b] < 1) { free(depths); return -1; }
+    depths[b] = d3o_depth(m->c.n_layers, alpha, gen_index[b]);
+  }
+  int32_t rc = step_with_depths(m, B, slots, tokens, depths, logits, hidden, trace);
+  free(depths);
+  return rc;
+}
+
+/* The same step with the retained count of every row given by the caller
+ * (0 <= depths[b] <= L): whatever schedule produced the counts, the window, the
+ * carried hidden state and the KV fill follow the rules above. */
+int32_t d3o_decode_step_depths(d3o_model *m, int32_t B, const int32_t *slots, const int32_t *tokens,
+                               const int32_t *depths, double *logits, double *hidden,
+                               double *trace) {
+  if (B < 1) return -1;
+  for (int b = 0; b < B; ++b)
+    if (depths[b] < 0 || depths[b] > m->c.n_layers) return -1;
+  return step_with_depths(m, B, slots, tokens, depths, logits, hidden, trace);
+}
+
+static int32_t step_with_depths(d3o_model *m, int32_t B, const int32_t *slots, const int32_t *tokens,
+                                const int32_t *depths, double *logits, double *hidden,
+                                double *trace) {
   const d3o_config *c = &m->c;
   int L = c->n_layers, d = c->d_model;
-  if (B < 1 || !(alpha > 0.0) || !(alpha <= 1.0)) return -1;
   for (int b = 0; b < B; ++b) {
     if (slots[b] < 0 || slots[b] >= c->max_slots) return -1;
-    if (tokens[b] < 0 || tokens[b] >= c->vocab || gen_index[b] < 1) return -1;
+    if (tokens[b] < 0 || tokens[b] >= c->vocab) return -1;
     if (m->pos[slots[b]] < 1) return -3;
     if (m->pos[slots[b]] >= c->max_seq) return -2;
     for (int a = 0; a < b; ++a)
@@ -490,7 +551,7 @@ int32_t d3o_decode_step(d3o_model *m, int32_t B, const int32_t *slots, const int
   for (int b = 0; b < B; ++b) {
     int slot = slots[b], pos = m->pos[slot];
     int32_t lo, hi;
-    int32_t n = d3o_window(L, alpha, gen_index[b], c->start_id, c->anchor, &lo, &hi);
+    int32_t n = window_of_depth(L, depths[b], c->start_id, c->anchor, &lo, &hi);
     if (n < 0) { free(x); return -1; }
     embed(m, tokens[b], x);
     for (int l = 0; l < L; ++l) {

@@ -151,6 +151,52 @@ def test_scheduled_step_equals_hand_truncated_stack(anchor, start):
         assert 0 in seen          # depth 0: logits of the bare embedding
 
 
+@pytest.mark.parametrize("anchor,start,fill", [(O.ANCHOR_START, 1, O.FILL_COPY), (O.ANCHOR_START, 0, O.FILL_NONE),
+                                               (O.ANCHOR_TAIL, 0, O.FILL_RECOMPUTE)])
+def test_step_with_given_depths_equals_the_alpha_step_and_the_truncated_stack(anchor, start, fill):
+    # (a) depths = floor(L alpha^i) must reproduce the alpha step bit for bit (logits, hidden,
+    #     cache); (b) any other depth sequence (here: linear decay) must equal the stack with
+    #     the window's blocks removed by hand.
+    shape = I.TINY_GQA
+    w = I.make_weights(shape, SEED + 6, gain_jitter=0.1)
+    toks = I.prompt_tokens(shape, SEED + 6, 0, 48).numpy()
+    L, alpha = shape.n_layers, 0.92
+    a = O.Oracle(shape, w, 2, 64, start_id=start, anchor=anchor, kv_fill=fill)
+    b = O.Oracle(shape, w, 2, 64, start_id=start, anchor=anchor, kv_fill=fill)
+    for orc in (a, b):
+        orc.prefill(0, toks[:5])
+        orc.prefill(1, toks[:9])
+    for i in range(1, 20):
+        gi = [i, i + 4]
+        tk = [int(toks[10 + i]), int(toks[20 + i])]
+        ra = a.decode_step([0, 1], tk, gi, alpha)
+        rb = b.decode_step_depths([0, 1], tk, [O.depth(L, alpha, g) for g in gi])
+        assert np.array_equal(ra["logits"], rb["logits"]) and np.array_equal(ra["hidden"], rb["hidden"])
+    for l in range(L):
+        for slot in (0, 1):
+            ka, va = a.read_kv(l, slot, a.slot_pos(slot) - 1)
+            kb, vb = b.read_kv(l, slot, b.slot_pos(slot) - 1)
+            assert np.array_equal(ka, kb, equal_nan=True) and np.array_equal(va, vb, equal_nan=True)
+    # (b) linear decay, one row, against the hand-truncated stack (nothing filled on that side)
+    c = O.Oracle(shape, w, 1, 64, start_id=start, anchor=anchor, kv_fill=O.FILL_NONE)
+    d = O.Oracle(shape, w, 1, 64)
+    c.prefill(0, toks[:6])
+    d.prefill(0, toks[:6])
+    seen = set()
+    for i in range(1, 16):
+        n = O.depth_linear(L, 1, 12, i)
+        nn, lo, hi = O.window_of_depth(L, n, start, anchor)
+        seen.add(nn)
+        keep = [l for l in range(L) if not (lo <= l < hi)]
+        tok = int(toks[6 + i])
+        r = c.decode_step_depths([0], [tok], [n])
+        lg, hid = d.decode_layers(0, tok, keep)
+        assert np.array_equal(r["logits"][0], lg) and np.array_equal(r["hidden"][0], hid)
+    assert len(seen) >= 3
+    with pytest.raises(ValueError):
+        c.decode_step_depths([0], [1], [L + 1])
+
+
 @pytest.mark.parametrize("anchor", [O.ANCHOR_START, O.ANCHOR_TAIL])
 def test_logits_do_not_depend_on_the_fill_mode(anchor):
     # depth never grows along a sequence, so no later token reads an entry that

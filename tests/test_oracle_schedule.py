@@ -110,3 +110,37 @@ def test_batch_schedule_against_brute_force(anchor):
             for l in range(L):
                 act = {b for b in range(B) if not (sch["lo"][b] <= l < sch["hi"][b])}
                 assert act == set(want_perm[:m[l]])
+
+
+# ---------------------------------------------------- linear decay between two bounds
+
+@pytest.mark.parametrize("upper,lower,span", [(32, 8, 255), (40, 14, 512), (80, 48, 100), (4, 0, 3),
+                                              (7, 7, 10), (32, 31, 1000)])
+def test_linear_depth_end_points_monotonicity_and_floor_sum(upper, lower, span):
+    # Sec. 3.4 / Sec. 4.1: linear decay between an upper and a lower bound of executed layers.
+    ns = [O.depth_linear(upper, lower, span, i) for i in range(span + 20)]
+    assert ns[0] == upper and ns[span] == lower and all(n == lower for n in ns[span:])
+    assert all(a >= b for a, b in zip(ns, ns[1:]))                     # never grows
+    assert all(0 <= a - b <= max(1, -(-(upper - lower) // span)) for a, b in zip(ns, ns[1:]))
+    # layers dropped over i = 0 .. span-1: the classical floor-sum identity
+    #   sum_{i<n} floor(a i / n) = ((a - 1)(n - 1) + gcd(a, n) - 1) / 2      (a, n >= 1)
+    a, n = upper - lower, span
+    dropped = sum(upper - v for v in ns[:span])
+    want = 0 if a == 0 else ((a - 1) * (n - 1) + math.gcd(a, n) - 1) // 2
+    assert dropped == want
+    # hence the mean retained count, the figure a target speed-up fixes
+    assert Fraction(sum(ns[:span]), span) == upper - Fraction(want, span)
+
+
+def test_linear_depth_rejects_bad_arguments():
+    for args in [(-1, 0, 5, 0), (4, 5, 5, 0), (4, -1, 5, 0), (4, 0, 0, 0), (4, 0, 5, -1)]:
+        assert O.depth_linear(*args) == -1
+
+
+def test_window_of_a_given_depth_is_the_window_of_the_rule():
+    L = 32
+    for alpha in (0.9, 0.99, 0.999):
+        for s, anchor in ((0, O.ANCHOR_START), (6, O.ANCHOR_START), (0, O.ANCHOR_TAIL)):
+            for i in (0, 1, 7, 50, 300, 4000):
+                assert O.window_of_depth(L, O.depth(L, alpha, i), s, anchor) == O.window(L, alpha, i, s, anchor)
+    assert O.window_of_depth(L, L + 1, 0)[0] == -1 and O.window_of_depth(L, -1, 0)[0] == -1
