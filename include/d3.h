@@ -166,6 +166,26 @@ int32_t d3_decode_step(d3_model *m, int32_t batch, const int32_t *slots, const i
                        const int32_t *gen_index, double alpha, float *logits_dev,
                        d3_step_stats *stats, const int32_t *tokens_dev);
 
+/* The same step with the retained block count of every row given by the caller
+ * instead of derived from (alpha, i): depths[b] in 0..L.  Window (anchor,
+ * start_id clamp), carried hidden state and KV fill follow the model's
+ * configuration exactly as in d3_decode_step, and d3_decode_step(alpha, i) is
+ * this call with depths[b] = d3_depth(L, alpha, i_b).  It serves the other
+ * schedules the paper discusses (Sec. 3.4, Sec. 4.1 "Comparison Methods"):
+ * linear decay between two bounds (d3_depth_linear), the Early-Exit direction
+ * (anchor TAIL), per-task tables, or a controller outside the library. */
+int32_t d3_decode_step_depths(d3_model *m, int32_t batch, const int32_t *slots, const int32_t *tokens,
+                              const int32_t *depths, float *logits_dev, d3_step_stats *stats,
+                              const int32_t *tokens_dev);
+
+/* Linear decay of the retained count between an upper and a lower bound (the
+ * shape Sec. 3.4 and Sec. 4.1 ascribe to SkipDecode; its constants are not in
+ * the paper, so they are arguments): upper at i = 0, lower from i = span on,
+ *   n(i) = upper - floor((upper - lower) * min(i, span) / span).
+ * Host, pure, integers only.  0 <= lower <= upper, span >= 1, i >= 0; otherwise
+ * D3_EINVAL. */
+int32_t d3_depth_linear(int32_t upper, int32_t lower, int64_t span, int64_t i);
+
 /* argmax over each row of logits_dev [batch][vocab], lowest index on ties
  * (greedy choice: Sec. 3.2, footnote on lm_head) -> tokens_dev [batch] int32. */
 int32_t d3_argmax(d3_model *m, const float *logits_dev, int32_t batch, int32_t *tokens_dev);

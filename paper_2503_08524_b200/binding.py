@@ -24,7 +24,7 @@ KV_CONTIGUOUS, KV_PAGED = 0, 1
 MAX_BATCH = 64     # D3_MAX_BATCH
 
 EXPORTS = ("d3_depth", "d3_schedule", "d3_workspace_bytes", "d3_load", "d3_prefill",
-           "d3_decode_step", "d3_argmax", "d3_read_schedule", "d3_read_hidden", "d3_read_kv",
+           "d3_decode_step", "d3_decode_step_depths", "d3_depth_linear", "d3_argmax", "d3_read_schedule", "d3_read_hidden", "d3_read_kv",
            "d3_set_exec", "d3_profile", "d3_read_profile", "d3_profile_name", "d3_read_fused_phases", "d3_decode_step_noalloc", "d3_slot_pos",
            "d3_kv_pages_used", "d3_reset_slot", "d3_sync", "d3_free", "d3_strerror")
 
@@ -69,6 +69,8 @@ def _load() -> C.CDLL:
     lib.d3_load.argtypes = [C.POINTER(Config), C.POINTER(Weights), P, P, P, C.POINTER(P)]
     lib.d3_prefill.argtypes = [P, I32, P, I32, P]
     lib.d3_decode_step.argtypes = [P, I32, P, P, P, C.c_double, P, C.POINTER(StepStats), P]
+    lib.d3_decode_step_depths.argtypes = [P, I32, P, P, P, P, C.POINTER(StepStats), P]
+    lib.d3_depth_linear.argtypes = [I32, I32, I64, I64]
     lib.d3_argmax.argtypes = [P, P, I32, P]
     lib.d3_read_schedule.argtypes = [P, P, P, P, P]
     lib.d3_read_hidden.argtypes = [P, P]
@@ -103,6 +105,11 @@ def strerror(code: int) -> str:
 def d3_depth(L: int, alpha: float, i: int) -> int:
     """floor(L * alpha^i); negative error code on bad arguments."""
     return int(LIB.d3_depth(L, alpha, i))
+
+
+def d3_depth_linear(upper: int, lower: int, span: int, i: int) -> int:
+    """upper - floor((upper - lower) * min(i, span) / span); negative error code on bad arguments."""
+    return int(LIB.d3_depth_linear(upper, lower, span, i))
 
 
 def d3_schedule(L: int, alpha: float, start_id: int, anchor: int, gen_index: Sequence[int]) -> Dict:
@@ -225,9 +232,15 @@ class D3Model:
             raise D3Error(rc, "d3_prefill")
         return logits
 
-    def d3_decode_step(self, slots, tokens, gen_index, alpha: float,
+    def d3_decode_step_depths(self, slots, tokens, depths, logits: Optional[torch.Tensor] = None,
+                              want_stats: bool = False, tokens_dev: Optional[torch.Tensor] = None):
+        """d3_decode_step with the retained block count of every row given by the caller."""
+        return self.d3_decode_step(slots, tokens, depths, None, logits, want_stats, tokens_dev)
+
+    def d3_decode_step(self, slots, tokens, gen_index, alpha: Optional[float],
                        logits: Optional[torch.Tensor] = None, want_stats: bool = False,
                        tokens_dev: Optional[torch.Tensor] = None):
+        """alpha None: `gen_index` holds retained block counts (d3_decode_step_depths)."""
         B = len(slots)
         s = np.ascontiguousarray(np.asarray(slots, dtype=np.int32))
         g = np.ascontiguousarray(np.asarray(gen_index, dtype=np.int32))
@@ -240,10 +253,16 @@ class D3Model:
             m = np.zeros(self.shape.n_layers, np.int32)
             st = StepStats(n.ctypes.data_as(C.POINTER(C.c_int32)), m.ctypes.data_as(C.POINTER(C.c_int32)),
                            0, 0, 0, 0)
-        rc = LIB.d3_decode_step(self.h, B, s.ctypes.data, None if t is None else t.ctypes.data,
-                                g.ctypes.data, float(alpha), logits.data_ptr(),
-                                C.byref(st) if st is not None else None,
-                                None if tokens_dev is None else tokens_dev.data_ptr())
+        if alpha is None:
+            rc = LIB.d3_decode_step_depths(self.h, B, s.ctypes.data, None if t is None else t.ctypes.data,
+                                           g.ctypes.data, logits.data_ptr(),
+                                           C.byref(st) if st is not None else None,
+                                           None if tokens_dev is None else tokens_dev.data_ptr())
+        else:
+            rc = LIB.d3_decode_step(self.h, B, s.ctypes.data, None if t is None else t.ctypes.data,
+                                    g.ctypes.data, float(alpha), logits.data_ptr(),
+                                    C.byref(st) if st is not None else None,
+                                    None if tokens_dev is None else tokens_dev.data_ptr())
         if rc != OK:
             raise D3Error(rc, "d3_decode_step")
         if want_stats:

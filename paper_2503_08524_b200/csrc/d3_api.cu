@@ -381,6 +381,10 @@ static int32_t run_fused_step(d3_model *m, const StepArgs &a, float *logits_dev,
   return (rc == 1 && cudaGetLastError() == cudaSuccess) ? D3_OK : D3_ECUDA;
 }
 
+static void schedule_of_depths(int32_t L, int32_t start_id, int32_t anchor, int32_t batch,
+                               const int32_t *depth, int32_t *n, int32_t *lo, int32_t *hi, int32_t *perm,
+                               int32_t *m_per_layer, int64_t *rows_layers, int32_t *layers_touched);
+
 // Paged layout: take back every page of `slot` (host list + device table, in stream order).
 static int32_t release_pages(d3_model *m, int32_t slot) {
   const d3_config &c = m->cfg;
@@ -414,8 +418,21 @@ int32_t d3_schedule(int32_t L, double alpha, int32_t start_id, int32_t anchor, i
     return D3_EINVAL;
   for (int b = 0; b < batch; ++b)
     if (gen_index[b] < 0) return D3_EINVAL;
+  int32_t depth[D3_MAX_BATCH];
+  for (int b = 0; b < batch; ++b) depth[b] = depth_host(L, alpha, gen_index[b]);
+  schedule_of_depths(L, start_id, anchor, batch, depth, n, lo, hi, perm, m_per_layer, rows_layers,
+                     layers_touched);
+  return D3_OK;
+}
+
+}  // extern "C"
+
+// Windows, depth-sorted order and per-block row counts for rows with the given depths.
+static void schedule_of_depths(int32_t L, int32_t start_id, int32_t anchor, int32_t batch,
+                               const int32_t *depth, int32_t *n, int32_t *lo, int32_t *hi, int32_t *perm,
+                               int32_t *m_per_layer, int64_t *rows_layers, int32_t *layers_touched) {
   for (int b = 0; b < batch; ++b) {
-    int32_t nb = depth_host(L, alpha, gen_index[b]);
+    int32_t nb = depth[b];
     if (anchor == D3_ANCHOR_TAIL) {
       lo[b] = nb; hi[b] = L;
     } else {
@@ -441,8 +458,9 @@ int32_t d3_schedule(int32_t L, double alpha, int32_t start_id, int32_t anchor, i
   }
   if (rows_layers) *rows_layers = tot;
   if (layers_touched) *layers_touched = touched;
-  return D3_OK;
 }
+
+extern "C" {
 
 int32_t d3_workspace_bytes(const d3_config *cfg, size_t *kv_bytes, size_t *scratch_bytes) {
   if (!config_ok(cfg) || !kv_bytes || !scratch_bytes) return D3_EINVAL;
@@ -607,15 +625,15 @@ int32_t d3_prefill(d3_model *m, int32_t slot, const int32_t *tokens, int32_t n_t
   return D3_OK;
 }
 
-int32_t d3_decode_step(d3_model *m, int32_t batch, const int32_t *slots, const int32_t *tokens,
-                       const int32_t *gen_index, double alpha, float *logits_dev,
-                       d3_step_stats *stats, const int32_t *tokens_dev) {
-  if (!m || !slots || !gen_index || !logits_dev || (!tokens && !tokens_dev)) return D3_EINVAL;
-  if (batch < 1 || !alpha_ok(alpha)) return D3_EINVAL;
-  if (batch > m->cfg.max_batch) return D3_ECAPACITY;
+// One generation step over rows whose retained counts `depth_in` are known.  `thr` / `gi`
+// are what the device derives the same counts from: the alpha thresholds with the
+// generation indices, or thr[k] = k with gi = L - depth (then #{k : gi < thr[k]} = depth).
+static int32_t decode_rows(d3_model *m, int32_t batch, const int32_t *slots, const int32_t *tokens,
+                           const int32_t *depth_in, const int32_t *thr, const int32_t *gi,
+                           float *logits_dev, d3_step_stats *stats, const int32_t *tokens_dev) {
   const d3_config &c = m->cfg;
   for (int b = 0; b < batch; ++b) {
-    if (slots[b] < 0 || slots[b] >= c.max_slots || gen_index[b] < 1) return D3_EINVAL;
+    if (slots[b] < 0 || slots[b] >= c.max_slots) return D3_EINVAL;
     if (!tokens_dev && (tokens[b] < 0 || tokens[b] >= c.vocab)) return D3_EINVAL;
   }
   for (int b = 0; b < batch; ++b) {
@@ -630,22 +648,20 @@ int32_t d3_decode_step(d3_model *m, int32_t batch, const int32_t *slots, const i
   StepArgs a;
   memset(&a, 0, sizeof(a));
   a.B = batch; a.L = L; a.start_id = c.start_id; a.anchor = c.anchor; a.tok_dev = tokens_dev;
-  memcpy(a.thr, thr_for(m, alpha), sizeof(a.thr));
+  memcpy(a.thr, thr, sizeof(a.thr));
   for (int b = 0; b < batch; ++b) {
-    a.slot[b] = slots[b]; a.tok[b] = tokens_dev ? 0 : tokens[b]; a.gi[b] = gen_index[b];
+    a.slot[b] = slots[b]; a.tok[b] = tokens_dev ? 0 : tokens[b]; a.gi[b] = gi[b];
     a.pos[b] = m->pos[slots[b]];
   }
   int32_t n[D3_MAX_BATCH], lo[D3_MAX_BATCH], hi[D3_MAX_BATCH], perm[D3_MAX_BATCH], m_l[D3_MAX_LAYERS];
   int64_t rows_layers = 0;
   int32_t touched = 0;
-  int32_t rc = d3_schedule(L, alpha, c.start_id, c.anchor, batch, gen_index, n, lo, hi, perm, m_l,
-                           &rows_layers, &touched);
-  if (rc != D3_OK) return rc;
+  schedule_of_depths(L, c.start_id, c.anchor, batch, depth_in, n, lo, hi, perm, m_l, &rows_layers, &touched);
   int32_t launches = 0;
   const bool fused = batch == 1 && m->fused_ok && m->exec_mode == D3_EXEC_AUTO &&
                      c.kv_fill != D3_FILL_RECOMPUTE;
-  rc = fused ? run_fused_step(m, a, logits_dev, &launches)
-             : run_step(m, a, n, lo, hi, perm, m_l, logits_dev, ROWS_ALL, &launches);
+  int32_t rc = fused ? run_fused_step(m, a, logits_dev, &launches)
+                     : run_step(m, a, n, lo, hi, perm, m_l, logits_dev, ROWS_ALL, &launches);
   if (rc != D3_OK) return rc;
   if (stats) {
     if (stats->n) memcpy(stats->n, n, sizeof(int32_t) * batch);
@@ -665,6 +681,43 @@ int32_t d3_decode_step(d3_model *m, int32_t batch, const int32_t *slots, const i
   }
   for (int b = 0; b < batch; ++b) m->pos[slots[b]] += 1;
   return D3_OK;
+}
+
+int32_t d3_decode_step(d3_model *m, int32_t batch, const int32_t *slots, const int32_t *tokens,
+                       const int32_t *gen_index, double alpha, float *logits_dev,
+                       d3_step_stats *stats, const int32_t *tokens_dev) {
+  if (!m || !slots || !gen_index || !logits_dev || (!tokens && !tokens_dev)) return D3_EINVAL;
+  if (batch < 1 || !alpha_ok(alpha)) return D3_EINVAL;
+  if (batch > m->cfg.max_batch) return D3_ECAPACITY;
+  int32_t depth[D3_MAX_BATCH];
+  for (int b = 0; b < batch; ++b) {
+    if (gen_index[b] < 1) return D3_EINVAL;
+    depth[b] = depth_host(m->cfg.n_layers, alpha, gen_index[b]);
+  }
+  return decode_rows(m, batch, slots, tokens, depth, thr_for(m, alpha), gen_index, logits_dev, stats,
+                     tokens_dev);
+}
+
+int32_t d3_decode_step_depths(d3_model *m, int32_t batch, const int32_t *slots, const int32_t *tokens,
+                              const int32_t *depths, float *logits_dev, d3_step_stats *stats,
+                              const int32_t *tokens_dev) {
+  if (!m || !slots || !depths || !logits_dev || (!tokens && !tokens_dev)) return D3_EINVAL;
+  if (batch < 1) return D3_EINVAL;
+  if (batch > m->cfg.max_batch) return D3_ECAPACITY;
+  const int L = m->cfg.n_layers;
+  int32_t thr[D3_MAX_LAYERS + 1], gi[D3_MAX_BATCH];
+  for (int k = 0; k <= D3_MAX_LAYERS; ++k) thr[k] = k;
+  for (int b = 0; b < batch; ++b) {
+    if (depths[b] < 0 || depths[b] > L) return D3_EINVAL;
+    gi[b] = L - depths[b];
+  }
+  return decode_rows(m, batch, slots, tokens, depths, thr, gi, logits_dev, stats, tokens_dev);
+}
+
+int32_t d3_depth_linear(int32_t upper, int32_t lower, int64_t span, int64_t i) {
+  if (upper < 0 || lower < 0 || lower > upper || span < 1 || i < 0) return D3_EINVAL;
+  const int64_t t = i < span ? i : span;
+  return (int32_t)(upper - ((int64_t)(upper - lower) * t) / span);
 }
 
 int32_t d3_argmax(d3_model *m, const float *logits_dev, int32_t batch, int32_t *tokens_dev) {

@@ -274,6 +274,49 @@ def test_production_widths(B, base, layers, Bn):
     gpu.close()
 
 
+# ------------------------------------------------ depths given by the caller
+
+@pytest.mark.parametrize("anchor,start,fill", [(0, 1, 1), (0, 0, 0), (1, 0, 2)])
+def test_steps_with_given_depths_linear_decay(B, anchor, start, fill):
+    # d3_decode_step_depths: the retained count of every row comes from the caller, here from the
+    # linear-decay rule (Sec. 3.4 / 4.1).  A batch of 5 rows at staggered indices (sequence of
+    # kernels, tensor-core projections) and a single row (single-kernel step), against the oracle.
+    shape = I.TINY_GQA
+    L, Bn = shape.n_layers, 5
+    orc, gpu = make_pair(shape, SEED + 12, 6, 96, 8, start_id=start, anchor=anchor, kv_fill=fill)
+    lens = I.uniform_ints(SEED + 12, 1, Bn + 1, 3, 30)
+    for b in range(Bn + 1):
+        p = I.prompt_tokens(shape, SEED + 12, b, lens[b]).numpy()
+        orc.prefill(b, p)
+        gpu.d3_prefill(b, p)
+    seen = set()
+    for step in range(14):
+        depths = [O.depth_linear(L, 1, 12, 1 + step + 3 * b) for b in range(Bn)]
+        assert depths == [B.d3_depth_linear(L, 1, 12, 1 + step + 3 * b) for b in range(Bn)]
+        toks = I.token_ids(SEED + 12, 300 + step, Bn + 1, shape.vocab).numpy()
+        r = orc.decode_step_depths(list(range(Bn)), toks[:Bn], depths)
+        g, st = gpu.d3_decode_step_depths(list(range(Bn)), toks[:Bn], depths, want_stats=True)
+        check_step(f"batch step {step}", g.cpu().numpy(), gpu.d3_read_hidden(Bn), r["logits"], r["hidden"])
+        want = [O.window_of_depth(L, d, start, anchor)[0] for d in depths]
+        assert list(st["n"]) == want and st["rows_layers"] == sum(want)
+        dev = gpu.d3_read_schedule(Bn)
+        assert list(dev["n"]) == want                     # the device derived the same counts
+        seen.update(want)
+        # one row alone: the single-kernel step (fill RECOMPUTE runs the kernel sequence)
+        d1 = O.depth_linear(L, 0, 9, step)
+        r1 = orc.decode_step_depths([Bn], [int(toks[Bn])], [d1])
+        g1, st1 = gpu.d3_decode_step_depths([Bn], [int(toks[Bn])], [d1], want_stats=True)
+        check_step(f"single step {step}", g1.cpu().numpy(), gpu.d3_read_hidden(1), r1["logits"], r1["hidden"])
+        assert st1["kernel_launches"] == 1 or fill == 2
+    assert len(seen) >= 3
+    for bad in ([L + 1], [-1]):
+        with pytest.raises(B.D3Error) as e:
+            gpu.d3_decode_step_depths([0], [1], bad)
+        assert e.value.code == B.EINVAL
+    gpu.d3_sync()
+    gpu.close()
+
+
 # ------------------------------------------------ the benchmark model at full depth
 
 def test_full_depth_7b_shape_against_oracle_and_between_paths(B):

@@ -116,3 +116,12 @@ def test_workspace_and_load_validation():
     assert B.LIB.d3_sync(None) == B.EINVAL and B.LIB.d3_slot_pos(None, 0) == B.EINVAL
     assert B.strerror(B.ESTATE) != B.strerror(B.ECAPACITY)
     assert B.strerror(-99) == "unknown error"
+
+
+def test_linear_depth_matches_the_oracle_rule():
+    for upper, lower, span in [(32, 8, 255), (40, 14, 512), (80, 48, 100), (4, 0, 3), (7, 7, 10)]:
+        for i in list(range(0, span + 5, max(1, span // 37))) + [span - 1, span, span + 1, 10 ** 9]:
+            assert B.d3_depth_linear(upper, lower, span, i) == O.depth_linear(upper, lower, span, i)
+    for bad in [(-1, 0, 5, 0), (4, 5, 5, 0), (4, -1, 5, 0), (4, 0, 0, 0), (4, 0, 5, -1)]:
+        assert B.d3_depth_linear(*bad) == B.EINVAL
+    assert B.LIB.d3_decode_step_depths(None, 1, None, None, None, None, None, None) == B.EINVAL
