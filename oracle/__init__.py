@@ -79,6 +79,8 @@ def _lib(kind: str) -> C.CDLL:
         lib.d3o_decode_step_depths.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p,
                                                C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         lib.d3o_depth_linear.argtypes = [C.c_int32, C.c_int32, C.c_int64, C.c_int64]
+        lib.d3o_probe.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(C.c_int32),
+                                  C.POINTER(C.c_double)]
         lib.d3o_window_of_depth.argtypes = [C.c_int32, C.c_int32, C.c_int32, C.c_int32,
                                             C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
         lib.d3o_decode_layers.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_int32,
@@ -246,6 +248,27 @@ class Oracle:
         if rc != 0:
             raise ValueError(f"oracle decode_step_depths failed ({rc})")
         return {"logits": logits, "hidden": hidden}
+
+    def probe(self, hidden):
+        """(token, confidence, logits) that lm_head(final_norm(hidden)) predicts."""
+        h = np.ascontiguousarray(np.asarray(hidden, dtype=np.float64))
+        logits = np.zeros(self.shape.vocab, np.float64)
+        tok, conf = C.c_int32(), C.c_double()
+        self.lib.d3o_probe(self.h, h.ctypes.data, logits.ctypes.data, C.byref(tok), C.byref(conf))
+        return int(tok.value), float(conf.value), logits
+
+    def saturation_probe(self, slots, tokens):
+        """One full-depth step; per row and block i = 1..L the token and confidence that
+        lm_head(h^i) predicts.  Returns dict(logits, hidden, tokens [B][L], conf [B][L])."""
+        L = self.shape.n_layers
+        r = self.decode_step(slots, tokens, [1] * len(slots), 1.0, want_trace=True)
+        toks = np.zeros((len(slots), L), np.int32)
+        conf = np.zeros((len(slots), L), np.float64)
+        for b in range(len(slots)):
+            for i in range(1, L + 1):
+                toks[b, i - 1], conf[b, i - 1], _ = self.probe(r["trace"][b, i])
+        r["tokens"], r["conf"] = toks, conf
+        return r
 
     def decode_layers(self, slot: int, token: int, layers: Sequence[int]):
         """One step over exactly the listed blocks (no schedule, no fill)."""

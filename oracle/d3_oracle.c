@@ -475,6 +475,28 @@ static void head(const d3o_model *m, const real *x, double *logits) {
   free(a); free(y);
 }
 
+/* Saturation probe (Sec. 3.2, the oracle experiment behind the saturation table):
+ * the token a block's output would predict, lm_head(h^i) with the model's final
+ * norm, and the confidence softmax gives it.  hidden [d] is a residual-stream
+ * state (e.g. a row of d3o_decode_step's trace); logits [vocab] is filled;
+ * *token = argmax (lowest index on ties), *confidence = its softmax probability. */
+int32_t d3o_probe(const d3o_model *m, const double *hidden, double *logits, int32_t *token,
+                  double *confidence) {
+  const d3o_config *c = &m->c;
+  real *x = (real *)malloc(sizeof(real) * (size_t)c->d_model);
+  for (int e = 0; e < c->d_model; ++e) x[e] = (real)hidden[e];
+  head(m, x, logits);
+  free(x);
+  int32_t best = 0;
+  for (int32_t r = 1; r < c->vocab; ++r)
+    if (logits[r] > logits[best]) best = r;
+  double z = 0.0;
+  for (int32_t r = 0; r < c->vocab; ++r) z += exp(logits[r] - logits[best]);
+  *token = best;
+  *confidence = 1.0 / z;
+  return 0;
+}
+
 /* Initiation phase (Sec. 3.1): every prompt token through all L blocks; the
  * logits of the last position choose T_0.  hidden_out (nullable, [d]) gets the
  * last position's residual stream before the final norm. */

@@ -78,6 +78,28 @@ def test_tail_truncation_equals_library_hidden_state(setup):
                 assert np.abs(r["trace"][0, k] - out.hidden_states[k][0, 20].numpy()).max() < HF_TOL
 
 
+def test_saturation_probe_equals_library_per_block_predictions(setup):
+    # Sec. 3.2: for the token at one position, what lm_head predicts from every block's output.
+    # The library gives the same from its hidden states: argmax and softmax of
+    # lm_head(norm(hidden_states[i])) for i < L, of its final logits for i = L.
+    shape, w, hf, cfg, toks, out = setup
+    L = shape.n_layers
+    orc = O.Oracle(shape, w, 1, 64)
+    orc.prefill(0, toks[:20].numpy())
+    r = orc.saturation_probe([0], [int(toks[20])])
+    assert orc.slot_pos(0) == 21 and r["tokens"].shape == (1, L)
+    for i in range(1, L + 1):
+        with torch.no_grad():
+            lg = (hf.lm_head(hf.model.norm(out.hidden_states[i][0, 20])) if i < L else out.logits[0, 20]).double()
+        p = torch.softmax(lg, -1)
+        assert r["tokens"][0, i - 1] == int(torch.argmax(lg))
+        assert abs(r["conf"][0, i - 1] - float(p.max())) < 1e-6
+    assert r["tokens"][0, L - 1] == O.argmax(r["logits"][0])
+    # closed form: a state whose logits are all equal has confidence 1 / vocab, token 0
+    tok, conf, lg = orc.probe(np.zeros(shape.d_model))
+    assert tok == 0 and abs(conf - 1.0 / shape.vocab) < 1e-12 and np.all(lg == 0.0)
+
+
 @pytest.mark.parametrize("anchor,start,alpha", [(O.ANCHOR_START, 1, 0.93), (O.ANCHOR_START, 2, 0.9),
                                                 (O.ANCHOR_TAIL, 0, 0.95), (O.ANCHOR_START, 3, 0.8)])
 @pytest.mark.parametrize("fill", [O.FILL_NONE, O.FILL_COPY, O.FILL_RECOMPUTE])
