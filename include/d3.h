@@ -178,6 +178,21 @@ int32_t d3_decode_step_depths(d3_model *m, int32_t batch, const int32_t *slots, 
                               const int32_t *depths, float *logits_dev, d3_step_stats *stats,
                               const int32_t *tokens_dev);
 
+/* Saturation probe (Sec. 3.2, the experiment behind the saturation table): one
+ * generation step at FULL depth for `batch` rows (slots advance and every
+ * block's K,V are cached as in a normal step) which, after every block i =
+ * 1..L, also runs the block's output through the final norm and the LM head
+ * and records what it would predict: block_tokens_dev[b][i-1] (DEVICE int32
+ * [batch][L]) = argmax, lowest index on ties; block_conf_dev[b][i-1] (DEVICE
+ * fp32 [batch][L], nullable) = the softmax probability of that token.  Column
+ * L-1 is the model's own prediction; a row's saturation depth is the first
+ * block from which the column agrees with it.  logits_dev [batch][vocab]
+ * (fp32) is used as the work buffer and ends up holding the final logits.
+ * Costs L LM-head projections ("without regard to cost", as the paper says);
+ * always runs as the sequence of kernels. */
+int32_t d3_saturation_probe(d3_model *m, int32_t batch, const int32_t *slots, const int32_t *tokens,
+                            float *logits_dev, int32_t *block_tokens_dev, float *block_conf_dev);
+
 /* Linear decay of the retained count between an upper and a lower bound (the
  * shape Sec. 3.4 and Sec. 4.1 ascribe to SkipDecode; its constants are not in
  * the paper, so they are arguments): upper at i = 0, lower from i = span on,

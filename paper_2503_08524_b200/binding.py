@@ -24,7 +24,8 @@ KV_CONTIGUOUS, KV_PAGED = 0, 1
 MAX_BATCH = 64     # D3_MAX_BATCH
 
 EXPORTS = ("d3_depth", "d3_schedule", "d3_workspace_bytes", "d3_load", "d3_prefill",
-           "d3_decode_step", "d3_decode_step_depths", "d3_depth_linear", "d3_argmax", "d3_read_schedule", "d3_read_hidden", "d3_read_kv",
+           "d3_decode_step", "d3_decode_step_depths", "d3_depth_linear", "d3_saturation_probe",
+           "d3_argmax", "d3_read_schedule", "d3_read_hidden", "d3_read_kv",
            "d3_set_exec", "d3_profile", "d3_read_profile", "d3_profile_name", "d3_read_fused_phases", "d3_decode_step_noalloc", "d3_slot_pos",
            "d3_kv_pages_used", "d3_reset_slot", "d3_sync", "d3_free", "d3_strerror")
 
@@ -71,6 +72,7 @@ def _load() -> C.CDLL:
     lib.d3_decode_step.argtypes = [P, I32, P, P, P, C.c_double, P, C.POINTER(StepStats), P]
     lib.d3_decode_step_depths.argtypes = [P, I32, P, P, P, P, C.POINTER(StepStats), P]
     lib.d3_depth_linear.argtypes = [I32, I32, I64, I64]
+    lib.d3_saturation_probe.argtypes = [P, I32, P, P, P, P, P]
     lib.d3_argmax.argtypes = [P, P, I32, P]
     lib.d3_read_schedule.argtypes = [P, P, P, P, P]
     lib.d3_read_hidden.argtypes = [P, P]
@@ -271,6 +273,21 @@ class D3Model:
                             "kernel_launches": int(st.kernel_launches),
                             "algorithmic_bytes": int(st.algorithmic_bytes)}
         return logits
+
+    def d3_saturation_probe(self, slots, tokens):
+        """One full-depth step; returns (logits [B][V], tokens [B][L] int32, conf [B][L] fp32),
+        all on the device: what the LM head predicts from every block's output."""
+        B, L = len(slots), self.shape.n_layers
+        s = np.ascontiguousarray(np.asarray(slots, dtype=np.int32))
+        t = np.ascontiguousarray(np.asarray(tokens, dtype=np.int32))
+        logits = torch.empty((B, self.shape.vocab), dtype=torch.float32, device=self.device)
+        toks = torch.empty((B, L), dtype=torch.int32, device=self.device)
+        conf = torch.empty((B, L), dtype=torch.float32, device=self.device)
+        rc = LIB.d3_saturation_probe(self.h, B, s.ctypes.data, t.ctypes.data, logits.data_ptr(),
+                                     toks.data_ptr(), conf.data_ptr())
+        if rc != OK:
+            raise D3Error(rc, "d3_saturation_probe")
+        return logits, toks, conf
 
     def d3_argmax(self, logits: torch.Tensor, out: Optional[torch.Tensor] = None) -> torch.Tensor:
         B = 1 if logits.dim() == 1 else logits.shape[0]

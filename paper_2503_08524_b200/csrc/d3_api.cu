@@ -248,9 +248,17 @@ static int project(d3_model *m, const GemvArgs &g, int epi, int rows) {
 // Enqueue one step over the rows described by `a` (already validated).
 // logits_mode: ROWS_ALL -> logits_dev[caller row][V]; ROWS_LAST -> logits_dev[V]
 // for the last row; logits_dev may be NULL (no LM head).
+// `probe` (nullable): after every block, the token and confidence the LM head predicts from the
+// block's output go to probe->tokens / conf [B][L] (device); logits_dev is the work buffer.
+struct ProbeOut {
+  int32_t *tokens;
+  float *conf;
+};
+
 static int32_t run_step(d3_model *m, const StepArgs &a, const int32_t *n, const int32_t *lo,
                         const int32_t *hi, const int32_t *perm, const int32_t *m_l,
-                        float *logits_dev, int logits_mode, int32_t *launches_out) {
+                        float *logits_dev, int logits_mode, int32_t *launches_out,
+                        const ProbeOut *probe = nullptr) {
   const d3_config &c = m->cfg;
   const Dims &dm = m->dm;
   cudaStream_t st = m->stream;
@@ -315,6 +323,17 @@ static int32_t run_step(d3_model *m, const StepArgs &a, const int32_t *n, const 
       g.act_stride = dm.f; g.gain = nullptr; g.out = m->x(); g.out_stride = dm.d;
       { ProfScope ps(m, PK_DOWN); launches += project(m, g, EPI_RESID, ml); }
     }
+    if (probe && logits_dev && l + 1 < L) {
+      // every row's state after block l through the final norm and the LM head (Sec. 3.2)
+      GemvArgs h = g;
+      h.layer = 0; h.row_mode = ROWS_ALL;
+      h.W = m->lm_head; h.W2 = nullptr; h.R = dm.V; h.K = dm.d; h.act = m->x(); h.act_stride = dm.d;
+      h.tmap_w = tm ? &m->tm_head : nullptr; h.tmap_w2 = nullptr;
+      h.gain = m->final_norm; h.out = logits_dev; h.out_stride = dm.V; h.out_col0 = 0;
+      ProfScope ps(m, PK_HEAD);
+      launches += project(m, h, EPI_LOGITS, B);
+      launches += launch_argmax_conf(logits_dev, B, dm.V, probe->tokens, probe->conf, L, l, st);
+    }
     if (c.kv_fill == D3_FILL_RECOMPUTE && ml < B) {
       // rows that drop block l: K,V from the block's own norm, W_k, W_v on the carried state
       g.row_mode = ROWS_SUFFIX;
@@ -340,6 +359,8 @@ static int32_t run_step(d3_model *m, const StepArgs &a, const int32_t *n, const 
     g.tmap_w = tm ? &m->tm_head : nullptr; g.tmap_w2 = nullptr;
     g.gain = m->final_norm; g.out = logits_dev; g.out_stride = dm.V; g.out_col0 = 0;
     { ProfScope ps(m, PK_HEAD); launches += project(m, g, EPI_LOGITS, logits_mode == ROWS_LAST ? 1 : B); }
+    if (probe)
+      launches += launch_argmax_conf(logits_dev, B, dm.V, probe->tokens, probe->conf, L, L - 1, st);
   }
   m->last_B = B;
   for (int b = 0; b < B; ++b) m->last_perm[b] = perm[b];
@@ -630,7 +651,8 @@ int32_t d3_prefill(d3_model *m, int32_t slot, const int32_t *tokens, int32_t n_t
 // generation indices, or thr[k] = k with gi = L - depth (then #{k : gi < thr[k]} = depth).
 static int32_t decode_rows(d3_model *m, int32_t batch, const int32_t *slots, const int32_t *tokens,
                            const int32_t *depth_in, const int32_t *thr, const int32_t *gi,
-                           float *logits_dev, d3_step_stats *stats, const int32_t *tokens_dev) {
+                           float *logits_dev, d3_step_stats *stats, const int32_t *tokens_dev,
+                           const ProbeOut *probe = nullptr) {
   const d3_config &c = m->cfg;
   for (int b = 0; b < batch; ++b) {
     if (slots[b] < 0 || slots[b] >= c.max_slots) return D3_EINVAL;
@@ -659,9 +681,9 @@ static int32_t decode_rows(d3_model *m, int32_t batch, const int32_t *slots, con
   schedule_of_depths(L, c.start_id, c.anchor, batch, depth_in, n, lo, hi, perm, m_l, &rows_layers, &touched);
   int32_t launches = 0;
   const bool fused = batch == 1 && m->fused_ok && m->exec_mode == D3_EXEC_AUTO &&
-                     c.kv_fill != D3_FILL_RECOMPUTE;
+                     c.kv_fill != D3_FILL_RECOMPUTE && !probe;
   int32_t rc = fused ? run_fused_step(m, a, logits_dev, &launches)
-                     : run_step(m, a, n, lo, hi, perm, m_l, logits_dev, ROWS_ALL, &launches);
+                     : run_step(m, a, n, lo, hi, perm, m_l, logits_dev, ROWS_ALL, &launches, probe);
   if (rc != D3_OK) return rc;
   if (stats) {
     if (stats->n) memcpy(stats->n, n, sizeof(int32_t) * batch);
@@ -712,6 +734,19 @@ int32_t d3_decode_step_depths(d3_model *m, int32_t batch, const int32_t *slots, 
     gi[b] = L - depths[b];
   }
   return decode_rows(m, batch, slots, tokens, depths, thr, gi, logits_dev, stats, tokens_dev);
+}
+
+int32_t d3_saturation_probe(d3_model *m, int32_t batch, const int32_t *slots, const int32_t *tokens,
+                            float *logits_dev, int32_t *block_tokens_dev, float *block_conf_dev) {
+  if (!m || !slots || !tokens || !logits_dev || !block_tokens_dev) return D3_EINVAL;
+  if (batch < 1) return D3_EINVAL;
+  if (batch > m->cfg.max_batch) return D3_ECAPACITY;
+  const int L = m->cfg.n_layers;
+  int32_t thr[D3_MAX_LAYERS + 1], gi[D3_MAX_BATCH], depth[D3_MAX_BATCH];
+  for (int k = 0; k <= D3_MAX_LAYERS; ++k) thr[k] = k;
+  for (int b = 0; b < batch; ++b) { gi[b] = 0; depth[b] = L; }   // every row at full depth
+  ProbeOut probe{block_tokens_dev, block_conf_dev};
+  return decode_rows(m, batch, slots, tokens, depth, thr, gi, logits_dev, nullptr, nullptr, &probe);
 }
 
 int32_t d3_depth_linear(int32_t upper, int32_t lower, int64_t span, int64_t i) {

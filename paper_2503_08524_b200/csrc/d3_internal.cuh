@@ -190,6 +190,8 @@ int launch_attention(const float *qkv, const bf16 *Kc, const bf16 *Vc, const Dev
                      float *part_ml, float *attn_out, const Dims &dm, cudaStream_t st);
 int launch_fill_copy(bf16 *Kc, bf16 *Vc, const DevSched *s, int B, const Dims &dm, cudaStream_t st);
 int launch_argmax(const float *logits, int B, int V, int32_t *out, cudaStream_t st);
+int launch_argmax_conf(const float *logits, int B, int V, int32_t *tok, float *conf, int stride, int col,
+                       cudaStream_t st);
 // paged KV cache: entries of the device block table that change before a step
 struct TableUpdate {
   static constexpr int kMax = 256;

@@ -641,6 +641,55 @@ __global__ void __launch_bounds__(1024) k_argmax(const float *logits, int V, int
   if (threadIdx.x == 0) out[blockIdx.x] = si[0] == 0x7fffffff ? 0 : si[0];
 }
 
+// argmax and its softmax probability of one logits row; results at out[row * stride + col]
+__global__ void __launch_bounds__(1024) k_argmax_conf(const float *logits, int V, int32_t *tok, float *conf,
+                                                      int stride, int col) {
+  pdl_wait();
+  pdl_trigger();
+  const float *p = logits + (size_t)blockIdx.x * V;
+  float best = -INFINITY;
+  int bi = 0x7fffffff;
+  for (int i = threadIdx.x; i < V; i += blockDim.x) {
+    float v = p[i];
+    if (v > best) { best = v; bi = i; }
+  }
+  __shared__ float sv[1024];
+  __shared__ int si[1024];
+  sv[threadIdx.x] = best; si[threadIdx.x] = bi;
+  __syncthreads();
+  for (int o = blockDim.x / 2; o > 0; o >>= 1) {
+    if (threadIdx.x < o) {
+      float v2 = sv[threadIdx.x + o];
+      int i2 = si[threadIdx.x + o];
+      if (v2 > sv[threadIdx.x] || (v2 == sv[threadIdx.x] && i2 < si[threadIdx.x])) {
+        sv[threadIdx.x] = v2; si[threadIdx.x] = i2;
+      }
+    }
+    __syncthreads();
+  }
+  const float mx = sv[0];
+  const int arg = si[0] == 0x7fffffff ? 0 : si[0];
+  __syncthreads();
+  float z = 0.f;
+  for (int i = threadIdx.x; i < V; i += blockDim.x) z += __expf(p[i] - mx);
+  sv[threadIdx.x] = z;
+  __syncthreads();
+  for (int o = blockDim.x / 2; o > 0; o >>= 1) {
+    if (threadIdx.x < o) sv[threadIdx.x] += sv[threadIdx.x + o];
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) {
+    tok[(size_t)blockIdx.x * stride + col] = arg;
+    if (conf) conf[(size_t)blockIdx.x * stride + col] = 1.f / sv[0];
+  }
+}
+
+int launch_argmax_conf(const float *logits, int B, int V, int32_t *tok, float *conf, int stride, int col,
+                       cudaStream_t st) {
+  launch_pdl(k_argmax_conf, dim3(B), dim3(1024), 0, st, logits, V, tok, conf, stride, col);
+  return 1;
+}
+
 int launch_argmax(const float *logits, int B, int V, int32_t *out, cudaStream_t st) {
   launch_pdl(k_argmax, dim3(B), dim3(1024), 0, st, logits, V, out);
   return 1;

@@ -317,6 +317,38 @@ def test_steps_with_given_depths_linear_decay(B, anchor, start, fill):
     gpu.close()
 
 
+# ------------------------------------------------ saturation probe
+
+@pytest.mark.parametrize("shape,Bn", [(I.TINY, 3), (I.TINY_GQA, 1)], ids=["mha-b3", "gqa-b1"])
+def test_saturation_probe_matches_oracle(B, shape, Bn):
+    # Sec. 3.2: per block, the token and confidence the LM head predicts from the block's output
+    L = shape.n_layers
+    orc, gpu = make_pair(shape, SEED + 13, Bn, 64, 4)
+    for b in range(Bn):
+        p = I.prompt_tokens(shape, SEED + 13, b, 5 + 4 * b).numpy()
+        orc.prefill(b, p)
+        gpu.d3_prefill(b, p)
+    for step in range(3):
+        toks = I.token_ids(SEED + 13, 50 + step, Bn, shape.vocab).numpy()
+        r = orc.saturation_probe(list(range(Bn)), toks)
+        lg, gt, gc = gpu.d3_saturation_probe(list(range(Bn)), toks)
+        check_step(f"step {step}", lg.cpu().numpy(), gpu.d3_read_hidden(Bn), r["logits"], r["hidden"])
+        gt, gc = gt.cpu().numpy(), gc.cpu().numpy()
+        for b in range(Bn):
+            assert gpu.d3_slot_pos(b) == orc.slot_pos(b)
+            for i in range(1, L + 1):
+                _, _, ol = orc.probe(r["trace"][b, i])
+                top = np.sort(ol)[-2:]
+                if top[1] - top[0] > 4 * LOGITS_MAX_ABS:          # not a near-tie
+                    assert gt[b, i - 1] == r["tokens"][b, i - 1], (b, i)
+                    assert abs(gc[b, i - 1] - r["conf"][b, i - 1]) <= 0.05 * r["conf"][b, i - 1] + 1e-6
+                else:                                              # either candidate is valid
+                    assert ol[gt[b, i - 1]] >= top[1] - 4 * LOGITS_MAX_ABS
+            assert gt[b, L - 1] == int(gpu.d3_argmax(lg)[b].item())
+    gpu.d3_sync()
+    gpu.close()
+
+
 # ------------------------------------------------ the benchmark model at full depth
 
 def test_full_depth_7b_shape_against_oracle_and_between_paths(B):
