@@ -220,10 +220,9 @@ def main():
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device(dev))
 
-    def barrier():
-        if dist is not None:
-            dist.barrier()
-        torch.cuda.synchronize()
+    from paper_2503_08524_b200.replicas import Replicas
+    reps = Replicas(dist, dev)
+    barrier = reps.barrier
 
     shape = I.LLAMA_7B if args.layers <= 0 else I.LLAMA_7B.with_layers(args.layers)
     start_id = int(START_FRACTION * shape.n_layers)
@@ -266,12 +265,7 @@ def main():
         model.d3_profile(False)
         return ms, tot, prof
 
-    def max_over_ranks(ms):
-        if dist is None:
-            return ms
-        t = torch.tensor([ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+    max_over_ranks = reps.max_ms
 
     # ---- main timed region (clock samples taken meanwhile)
     sampler = ClockSampler(local) if rank == 0 else None
