@@ -217,7 +217,8 @@ int32_t d3_read_kv(d3_model *m, int32_t layer, int32_t slot, int32_t pos, float 
 
 /* How decode steps execute.  AUTO: a batch of one row runs as a single persistent
  * cooperative kernel when the device and sizes allow it (fill modes NONE and
- * COPY), everything else as a sequence of kernels per block, whose projections
+ * COPY, contiguous cache, at most 512 MiB of weights per block: beyond that the
+ * kernel sequence measured as fast), everything else as a sequence of kernels per block, whose projections
  * run on the tensor cores (tcgen05, activations split exactly into three bf16 terms, fp32
  * accumulate) once the block's depth group has D3_TENSOR_MIN_ROWS rows or more and
  * as FP32-FMA GEMVs below that.  KERNELS: always the sequence of kernels with
@@ -227,6 +228,8 @@ int32_t d3_read_kv(d3_model *m, int32_t layer, int32_t slot, int32_t pos, float 
 #define D3_EXEC_AUTO 0
 #define D3_EXEC_KERNELS 1
 #define D3_EXEC_TENSOR 2
+#define D3_EXEC_FUSED 3    /* like AUTO, but a single row takes the single-kernel step whatever
+                              the block size (D3_EINVAL when that kernel cannot serve the model) */
 #define D3_TENSOR_MIN_ROWS 2
 int32_t d3_set_exec(d3_model *m, int32_t mode);
 

@@ -19,7 +19,7 @@ OK, EINVAL, ECAPACITY, ESTATE, ECUDA, ETIMEOUT = 0, -1, -2, -3, -4, -5
 ANCHOR_START, ANCHOR_TAIL = 0, 1
 FILL_NONE, FILL_COPY, FILL_RECOMPUTE = 0, 1, 2
 MAX_BATCH, MAX_LAYERS, PROF_KINDS = 64, 128, 22
-EXEC_AUTO, EXEC_KERNELS, EXEC_TENSOR = 0, 1, 2
+EXEC_AUTO, EXEC_KERNELS, EXEC_TENSOR, EXEC_FUSED = 0, 1, 2, 3
 KV_CONTIGUOUS, KV_PAGED = 0, 1
 MAX_BATCH = 64     # D3_MAX_BATCH
 

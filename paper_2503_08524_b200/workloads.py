@@ -1,7 +1,7 @@
 """Batched decode workloads (several sequences per step, mixed depths).
 
   python -m paper_2503_08524_b200.workloads c3|c4|c5 [--layers N] [--steps K] [--alpha A]
-                                                     [--exec auto|kernels|tensor] [--profile]
+                                                     [--exec auto|kernels|tensor] [--rows R] [--profile]
 
 The workloads follow the batched configurations the paper's runs suggest
 (static batches of a few sequences, prompts of a few hundred to ~1k tokens,
@@ -57,6 +57,7 @@ def main(argv=None) -> int:
     ap.add_argument("--alpha", type=float, default=0.0)
     ap.add_argument("--gen-offset", type=int, default=0, help="added to every row's generation index")
     ap.add_argument("--exec", dest="exec_mode", default="auto", choices=sorted(EXEC))
+    ap.add_argument("--rows", type=int, default=0, help="override the workload's row count (1 = single-kernel step)")
     ap.add_argument("--profile", action="store_true")
     args = ap.parse_args(argv)
 
@@ -64,6 +65,7 @@ def main(argv=None) -> int:
     if not torch.cuda.is_available():
         raise SystemExit("needs a CUDA device (no CPU fallback)")
     base, rows, plo, phi, stagger, alpha, steps = WORKLOADS[args.workload]
+    rows = args.rows if args.rows > 0 else rows
     shape = base.with_layers(args.layers) if args.layers > 0 else base
     alpha = args.alpha if args.alpha > 0 else alpha
     K, W = (args.steps if args.steps > 0 else steps), max(args.warmup, 3)

@@ -263,13 +263,18 @@ def test_production_widths(B, base, layers, Bn):
         o = orc.prefill(b, p)
         g = gpu.d3_prefill(b, p)
         check_step(f"prefill {b}", g.cpu().numpy()[None], None, o[None], None)
-    for step in range(3):
+    for step in range(4):
+        # single rows: the single-kernel step on even steps, whatever AUTO picks on odd ones
+        # (blocks above 512 MiB go to the tensor-core kernel sequence there)
+        gpu.d3_set_exec(B.EXEC_FUSED if (Bn == 1 and not pk and step % 2 == 0) else B.EXEC_AUTO)
         toks = I.token_ids(SEED + 5, 40 + step, Bn, shape.vocab).numpy()
         gi = [1 + step + 2 * b for b in range(Bn)]
         alpha = 0.8
         r = orc.decode_step(list(range(Bn)), toks, gi, alpha)
-        g = gpu.d3_decode_step(list(range(Bn)), toks, gi, alpha)
+        g, st = gpu.d3_decode_step(list(range(Bn)), toks, gi, alpha, want_stats=True)
         check_step(f"step {step}", g.cpu().numpy(), gpu.d3_read_hidden(Bn), r["logits"], r["hidden"])
+        if Bn == 1 and not pk and step % 2 == 0:
+            assert st["kernel_launches"] == 1
     gpu.d3_sync()          # raises on a deferred device status (a bounded wait that ran out)
     gpu.close()
 

@@ -1,5 +1,6 @@
 """The N > 1 bookkeeping of the benchmark (replicas only: no exchange on the data
 path), run as two gloo ranks on the CPU."""
+import json
 import os
 import socket
 
@@ -24,18 +25,18 @@ def _rank_main(rank, world, port, out):
     reps.barrier()
     ms_local = 10.0 + 5.0 * rank          # rank 1 is the slow one
     units_local = 255 * (rank + 1)        # unequal on purpose
-    out[rank] = (reps.rank, reps.world, reps.max_ms(ms_local), reps.total_units(units_local),
-                 reps.throughput(units_local, ms_local))
+    res = (reps.rank, reps.world, reps.max_ms(ms_local), reps.total_units(units_local),
+           reps.throughput(units_local, ms_local))
+    with open(os.path.join(out, f"rank{rank}.json"), "w") as f:
+        json.dump(res, f)
     reps.barrier()
     dist.destroy_process_group()
 
 
-def test_two_replicas_report_job_totals_over_the_slowest_rank():
+def test_two_replicas_report_job_totals_over_the_slowest_rank(tmp_path):
     world, port = 2, _free_port()
-    with mp.Manager() as mgr:
-        out = mgr.dict()
-        mp.spawn(_rank_main, args=(world, port, out), nprocs=world, join=True)
-        res = dict(out)
+    mp.spawn(_rank_main, args=(world, port, str(tmp_path)), nprocs=world, join=True)
+    res = {r: json.load(open(tmp_path / f"rank{r}.json")) for r in range(world)}
     for rank in range(world):
         r, w, ms, units, tput = res[rank]
         assert (r, w) == (rank, world)
