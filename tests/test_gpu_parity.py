@@ -279,6 +279,39 @@ def test_production_widths(B, base, layers, Bn):
     gpu.close()
 
 
+# ------------------------------------------------ the largest step the ABI allows
+
+def test_sixty_four_rows_per_step(B):
+    # D3_MAX_BATCH rows: the widest tensor-core operand (3 x 64 rows -> UMMA N = 192, 256 TMEM
+    # columns, two-stage ring), 64-position prefill passes, every depth from L - 1 down to 0 in one step
+    shape = I.TINY_GQA
+    Bn, L = 64, shape.n_layers
+    orc, gpu = make_pair(shape, SEED + 14, Bn, 160, Bn, start_id=0, kv_fill=1)
+    for b in range(Bn):
+        n = 1 + (37 * b) % 90                      # 1 .. 90 tokens: one or two passes, ragged
+        p = I.prompt_tokens(shape, SEED + 14, b, n).numpy()
+        o = orc.prefill(b, p)
+        g = gpu.d3_prefill(b, p)
+        if b % 8 == 0:
+            check_step(f"prefill {b}", g.cpu().numpy()[None], None, o[None], None)
+    seen = set()
+    for step in range(3):
+        toks = I.token_ids(SEED + 14, 70 + step, Bn, shape.vocab).numpy()
+        gi = [1 + step + b for b in range(Bn)]
+        r = orc.decode_step(list(range(Bn)), toks, gi, 0.955)
+        g, st = gpu.d3_decode_step(list(range(Bn)), toks, gi, 0.955, want_stats=True)
+        check_step(f"step {step}", g.cpu().numpy(), gpu.d3_read_hidden(Bn), r["logits"], r["hidden"])
+        want = O.schedule(L, 0.955, 0, 0, gi)
+        assert np.array_equal(st["n"], want["n"]) and np.array_equal(st["m_per_layer"], want["m_per_layer"])
+        seen.update(int(v) for v in st["n"])
+    assert seen == set(range(L))                    # floor(4 * 0.955^i): 3 down to 0
+    with pytest.raises(B.D3Error) as e:             # 65 rows: over the limit of the model
+        gpu.d3_decode_step(list(range(Bn)) + [0], [1] * 65, [1] * 65, 1.0)
+    assert e.value.code == B.ECAPACITY
+    gpu.d3_sync()
+    gpu.close()
+
+
 # ------------------------------------------------ depths given by the caller
 
 @pytest.mark.parametrize("anchor,start,fill", [(0, 1, 1), (0, 0, 0), (1, 0, 2)])
