@@ -1,6 +1,8 @@
 // CUDA kernels of the D3 decode step (sm_100a): depth schedule + sort,
 // embedding gather, fused RMSNorm + projection GEMVs, RoPE + KV append,
 // split-K flash-decoding attention with grouped KV heads, KV fill, argmax.
+#include <stdlib.h>
+
 #include "d3_internal.cuh"
 
 namespace d3 {
@@ -324,6 +326,7 @@ static cudaError_t gemv_attr() {
 }
 
 int init_kernel_attributes() {
+  if (init_attention_mma() != 0) return -1;
   cudaError_t e = cudaSuccess;
 #define D3_ATTR(MT)                                           \
   if (e == cudaSuccess) e = gemv_attr<MT, EPI_STORE>();       \
@@ -556,7 +559,11 @@ static void attn_launch(const float *qkv, const bf16 *Kc, const bf16 *Vc, const 
 int launch_attention(const float *qkv, const bf16 *Kc, const bf16 *Vc, const DevSched *s, int layer,
                      int m_rows, int split_len, int n_splits, int max_splits, float *part_o,
                      float *part_ml, float *attn_out, const Dims &dm, cudaStream_t st) {
-  if (dm.dh == 128)
+  static const bool fma_path = getenv("D3_ATTN_FMA") != nullptr;   // the scalar kernel, for comparison
+  if (!fma_path)
+    launch_attention_partial_mma(qkv, Kc, Vc, s, layer, m_rows, split_len, n_splits, max_splits, part_o,
+                                 part_ml, dm, st);
+  else if (dm.dh == 128)
     attn_launch<128>(qkv, Kc, Vc, s, layer, m_rows, split_len, n_splits, max_splits, part_o, part_ml, dm, st);
   else if (dm.dh == 64)
     attn_launch<64>(qkv, Kc, Vc, s, layer, m_rows, split_len, n_splits, max_splits, part_o, part_ml, dm, st);
