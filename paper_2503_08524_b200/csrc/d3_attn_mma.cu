@@ -105,11 +105,14 @@ k_attn_partial_mma(const float *qkv, const bf16 *Kc, const bf16 *Vc, const DevSc
     const int p0 = chunk_pos(c);
     if (p0 < t1) {
       constexpr int CPR = DH * 2 / 16;   // 16-byte pieces per row
+      // the 16 positions are consecutive rows of the cache (one page at most: p0 is a multiple
+      // of 16 and a page holds a power of two >= 16 positions): one offset per trip
+      const size_t base = kv_offset(dm, dm.block_table, layer, slot, kvh, p0);
+      const int rmax = t1 - 1 - p0;      // rows past the end repeat the last valid one
 #pragma unroll
       for (int i = 0; i < 16 * CPR / 32; ++i) {
         const int idx = i * 32 + lane, r = idx / CPR, cidx = idx % CPR;
-        const int pos = min(p0 + r, t1 - 1);
-        const size_t off = kv_offset(dm, dm.block_table, layer, slot, kvh, pos) + cidx * 8;
+        const size_t off = base + (size_t)(min(r, rmax) * DH + cidx * 8);
         const uint32_t dst =
             (uint32_t)__cvta_generic_to_shared(vbuf + buf * VStage<DH>::kBytes + r * VStage<DH>::kRowBytes + cidx * 16);
         asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(Kc + off) : "memory");
