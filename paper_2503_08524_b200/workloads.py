@@ -1,7 +1,7 @@
 """Batched decode workloads (several sequences per step, mixed depths).
 
   python -m paper_2503_08524_b200.workloads c3|c4|c5 [--layers N] [--steps K] [--alpha A]
-                                                     [--exec auto|kernels|tensor] [--rows R] [--profile]
+                                                     [--exec auto|kernels|tensor|fused] [--rows R] [--profile]
 
 The workloads follow the batched configurations the paper's runs suggest
 (static batches of a few sequences, prompts of a few hundred to ~1k tokens,
@@ -37,7 +37,7 @@ WORKLOADS = {
     "c4": (I.LLAMA_13B, 8, 1024, 1024, 0, 0.998, 64),
     "c5": (I.LLAMA_70B, 4, 512, 512, 0, 0.998, 32),
 }
-EXEC = {"auto": 0, "kernels": 1, "tensor": 2}
+EXEC = {"auto": 0, "kernels": 1, "tensor": 2, "fused": 3}
 
 
 def measured_hbm_gbs():
