@@ -312,6 +312,36 @@ def test_sixty_four_rows_per_step(B):
     gpu.close()
 
 
+# ------------------------------------------------ tensor-core attention, every variant
+
+@pytest.mark.parametrize("hq,hkv,dh", [(32, 32, 128), (32, 32, 64), (32, 16, 128), (32, 8, 32), (16, 4, 64),
+                                       (32, 32, 32)],
+                         ids=["mha-128", "mha-64", "gq2-128", "gq4-32", "gq4-64", "mha-32"])
+def test_tensor_core_attention_variants(B, hq, hkv, dh):
+    # Many heads on a narrow model: rows x heads exceeds the CTA target, so every (row, head group)
+    # takes ONE piece of 260-340 positions (several 16-position trips per warp, a ragged last
+    # trip) and the MHA variants take the tensor-core kernel too (it needs >= 256 positions per
+    # piece there).  Contexts differ per row; 20 rows; against the oracle.
+    shape = I.ModelShape(f"heads-{hq}-{hkv}-{dh}", 2, 256, hq, hkv, dh, 512, 1024)
+    Bn = 20
+    orc, gpu = make_pair(shape, SEED + 15, Bn, 352, 32, start_id=0)
+    lens = I.uniform_ints(SEED + 15, 2, Bn, 260, 335)
+    for b in range(Bn):
+        p = I.prompt_tokens(shape, SEED + 15, b, lens[b]).numpy()
+        o = orc.prefill(b, p)
+        g = gpu.d3_prefill(b, p)
+        if b % 5 == 0:
+            check_step(f"prefill {b}", g.cpu().numpy()[None], None, o[None], None)
+    for step in range(3):
+        toks = I.token_ids(SEED + 15, 20 + step, Bn, shape.vocab).numpy()
+        gi = [1 + step + b for b in range(Bn)]
+        r = orc.decode_step(list(range(Bn)), toks, gi, 0.97)
+        g = gpu.d3_decode_step(list(range(Bn)), toks, gi, 0.97)
+        check_step(f"step {step}", g.cpu().numpy(), gpu.d3_read_hidden(Bn), r["logits"], r["hidden"])
+    gpu.d3_sync()
+    gpu.close()
+
+
 # ------------------------------------------------ depths given by the caller
 
 @pytest.mark.parametrize("anchor,start,fill", [(0, 1, 1), (0, 0, 0), (1, 0, 2)])
