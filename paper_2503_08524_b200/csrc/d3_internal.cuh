@@ -191,7 +191,7 @@ int launch_attention(const float *qkv, const bf16 *Kc, const bf16 *Vc, const Dev
 int init_attention_mma();
 int launch_attention_partial_mma(const float *qkv, const bf16 *Kc, const bf16 *Vc, const DevSched *s, int layer,
                                  int m_rows, int split_len, int n_splits, int max_splits, float *part_o,
-                                 float *part_ml, const Dims &dm, cudaStream_t st);
+                                 float *part_ml, float *attn_out, const Dims &dm, cudaStream_t st);
 int launch_fill_copy(bf16 *Kc, bf16 *Vc, const DevSched *s, int B, const Dims &dm, cudaStream_t st);
 int launch_argmax(const float *logits, int B, int V, int32_t *out, cudaStream_t st);
 int launch_argmax_conf(const float *logits, int B, int V, int32_t *tok, float *conf, int stride, int col,

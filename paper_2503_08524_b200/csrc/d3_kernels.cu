@@ -564,10 +564,11 @@ int launch_attention(const float *qkv, const bf16 *Kc, const bf16 *Vc, const Dev
   // 16-position trips per warp to amortise, unless several query heads share the K/V fragments:
   // measured, one row of the 13B shape (15 splits of 96 positions) is 13 % slower with it.
   const bool shared_kv = (dm.Hq / dm.Hkv) % 2 == 0;
-  if (!fma_path && (shared_kv || split_len >= 256))
+  if (!fma_path && (shared_kv || split_len >= 256)) {
     launch_attention_partial_mma(qkv, Kc, Vc, s, layer, m_rows, split_len, n_splits, max_splits, part_o,
-                                 part_ml, dm, st);
-  else if (dm.dh == 128)
+                                 part_ml, n_splits == 1 ? attn_out : nullptr, dm, st);
+    if (n_splits == 1) return 1;   // every row and head in one piece: written directly
+  } else if (dm.dh == 128)
     attn_launch<128>(qkv, Kc, Vc, s, layer, m_rows, split_len, n_splits, max_splits, part_o, part_ml, dm, st);
   else if (dm.dh == 64)
     attn_launch<64>(qkv, Kc, Vc, s, layer, m_rows, split_len, n_splits, max_splits, part_o, part_ml, dm, st);
