@@ -591,17 +591,21 @@ __global__ void k_fill_copy(bf16 *Kc, bf16 *Vc, const DevSched *s, Dims dm) {
   const int lo = s->lo_s[row], hi = s->hi_s[row];
   if (l < lo || l >= hi) return;
   const int slot = s->slot_s[row], pos = s->pos_s[row];
-  const int n = dm.Hkv * dm.dh;
+  // 16-byte pieces (8 bf16; head_dim is a multiple of 32, every cache row 16-byte aligned)
+  const int per_head = dm.dh / 8, n = dm.Hkv * per_head;
   for (int i = threadIdx.x; i < n; i += blockDim.x) {
-    int h = i / dm.dh, e = i % dm.dh;
-    size_t dst = kv_offset(dm, dm.block_table, l, slot, h, pos) + e;
+    const int h = i / per_head, e = (i % per_head) * 8;
+    uint4 *kd = reinterpret_cast<uint4 *>(Kc + kv_offset(dm, dm.block_table, l, slot, h, pos) + e);
+    uint4 *vd = reinterpret_cast<uint4 *>(Vc + kv_offset(dm, dm.block_table, l, slot, h, pos) + e);
     if (lo == 0) {
-      Kc[dst] = __float2bfloat16_rn(0.f);
-      Vc[dst] = __float2bfloat16_rn(0.f);
+      *kd = make_uint4(0u, 0u, 0u, 0u);   // bf16 zero is all-zero bits
+      *vd = make_uint4(0u, 0u, 0u, 0u);
     } else {
-      size_t src = kv_offset(dm, dm.block_table, lo - 1, slot, h, pos) + e;
-      Kc[dst] = Kc[src];
-      Vc[dst] = Vc[src];
+      const size_t src = kv_offset(dm, dm.block_table, lo - 1, slot, h, pos) + e;
+      const uint4 kw = *reinterpret_cast<const uint4 *>(Kc + src);
+      const uint4 vw = *reinterpret_cast<const uint4 *>(Vc + src);
+      *kd = kw;
+      *vd = vw;
     }
   }
 }
