@@ -325,6 +325,17 @@ def rope(v, pos: int, base: float, real: str = "f64") -> np.ndarray:
     return va.astype(np.float64)
 
 
+def round_bf16(x, real: str = "f64") -> np.ndarray:
+    """The bf16 value nearest to each element (ties to even), as the oracle stores K and V
+    when `kv_round_bf16` is set."""
+    lib = _lib(real)
+    xa = _real_array(lib, x).ravel()
+    out = np.zeros_like(xa)
+    lib.d3o_round_bf16.argtypes = [C.c_void_p, C.c_int32, C.c_void_p]
+    lib.d3o_round_bf16(xa.ctypes.data, xa.size, out.ctypes.data)
+    return out.astype(np.float64)
+
+
 def softmax(s, real: str = "f64") -> np.ndarray:
     lib = _lib(real)
     sa = _real_array(lib, s).copy()

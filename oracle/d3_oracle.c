@@ -35,6 +35,10 @@
  *                       (itself pinned above); linear decay: end points, monotonicity
  *                       and the floor-sum identity sum_{i<n} floor(a i / n) =
  *                       ((a-1)(n-1) + gcd(a,n) - 1) / 2
+ *   bf16 cache storage  round_bf16: hand-listed bit patterns (ties both ways, carry
+ *                       into the exponent, subnormals, overflow, a value that
+ *                       rounding twice would get wrong) and a sweep against
+ *                       the library conversion of fp32 inputs
  * Parity unpinned: the VALUES that fill modes COPY / RECOMPUTE leave in the
  * cache when the caller raises alpha between steps (the paper never states
  * which rule D3 itself uses); only their own definitions below fix them.
@@ -97,18 +101,26 @@ static real bf16_to_real(uint16_t b) {
   return (real)f;
 }
 
-/* round-to-nearest-even to bf16 precision, returned widened */
+/* The bf16 value nearest to x, ties to the even significand, returned widened:
+ * ONE rounding of the value as it stands (a detour through fp32 would round
+ * twice).  bf16 = 8 significand bits, exponent range of fp32: for |x| in
+ * [2^e, 2^(e+1)) the spacing is 2^(e-7), below 2^-126 it stays 2^-133
+ * (subnormals), and what rounds to 2^128 or beyond is infinity.  Zeros,
+ * infinities and NaN pass through. */
 static real round_bf16(real x) {
-  float f = (float)x;
-  uint32_t u;
-  memcpy(&u, &f, 4);
-  if ((u & 0x7f800000u) != 0x7f800000u) {
-    uint32_t lsb = (u >> 16) & 1u;
-    u += 0x7fffu + lsb;
-  }
-  u &= 0xffff0000u;
-  memcpy(&f, &u, 4);
-  return (real)f;
+  double v = (double)x;
+  if (v == 0.0 || isnan(v) || isinf(v)) return x;
+  int e = ilogb(v);
+  if (e < -126) e = -126;
+  double quantum = ldexp(1.0, e - 7);
+  double r = nearbyint(v / quantum) * quantum; /* default rounding mode: nearest, ties to even */
+  if (fabs(r) >= ldexp(1.0, 128)) r = copysign(INFINITY, v);
+  return (real)r;
+}
+
+/* test access to the storage rounding */
+void d3o_round_bf16(const real *in, int32_t n, real *out) {
+  for (int32_t k = 0; k < n; ++k) out[k] = round_bf16(in[k]);
 }
 
 static size_t kv_index(const d3o_config *c, int l, int slot, int t) {

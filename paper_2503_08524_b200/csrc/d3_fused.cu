@@ -1022,6 +1022,10 @@ static bool try_plan(FusedPlan &pl, const d3_config &c) {
       per_sm < 1)
     return false;
   pl.grid = sms < kFusedMaxCtas ? sms : kFusedMaxCtas;
+  if (const char *env = getenv("D3_FUSED_CTAS")) {   // tuning knob: fewer CTAs than SMs
+    const int want = atoi(env);
+    if (want >= 8 && want < pl.grid) pl.grid = want;
+  }
   return true;
 }
 
