@@ -7,13 +7,17 @@ One "step" is one decode step of the whole hot path (schedule, every retained
 block, KV fill, final norm + LM head) for the batch.  The workload is the
 Llama-2-7B-shaped decoder (random-init bf16, seeded), batch 1, prompt 512
 uniform-random token ids, generate 256; the K timed steps take their generation
-indices i evenly over 1..255 (K = 255, the default, is the run itself).
+indices i evenly over 1..255 (K = 255, the default, is the run itself).  The
+timed region of K steps is repeated (--reps, default 5); the median repetition
+is the reported value, the best one rides along.
 
 Prints ONE JSON line: decode tokens/s (device-timed, inputs resident in HBM),
 the HBM roofline of the dominant kernel and of the whole step, the same metric
 end to end through the C ABI with host buffers, the alpha = 1 run of the same
-kernels, and the CPU oracle timed on the host cores as a baseline.
+kernels, time to first token of the prompt, the batched workloads C3 / C4, and
+the CPU oracle timed on the host cores as a baseline.
 `--impl reference` times the CPU oracle alone on a bounded sample.
+`--gpus N` without a torchrun environment starts the N replica processes itself.
 """
 from __future__ import annotations
 
@@ -70,7 +74,7 @@ class ClockSampler:
               "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
               "clocks_event_reasons.sw_power_cap")
 
-    def __init__(self, device_index: int):
+    def __init__(self, device_index: int, period_ms: int = 50):
         self.tmp = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
         sel = str(device_index)
         try:
@@ -80,7 +84,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", sel, "--query-gpu=" + self.FIELDS,
-                 "--format=csv,noheader,nounits", "-lms", "100"],
+                 "--format=csv,noheader,nounits", "-lms", str(period_ms)],
                 stdout=self.tmp, stderr=subprocess.DEVNULL)
         except Exception:
             self.proc = None
@@ -118,23 +122,35 @@ class ClockSampler:
         return out
 
 
-def time_oracle(shape, w_cpu, alpha, start_id, steps, warmup):
-    """CPU oracle on a bounded sample: ORACLE_PROMPT-token prefill (untimed), then
-    `steps` timed decode steps with the same generation indices as the GPU run."""
+ORACLE_STEPS, ORACLE_PASSES = 40, 2
+
+
+def oracle_steps(k):
+    """Timed oracle steps per pass for a run of k GPU steps (the same rule in both arms)."""
+    return max(8, min(int(k), ORACLE_STEPS))
+
+
+def time_oracle(shape, w_cpu, alpha, start_id, steps):
+    """CPU oracle on a bounded sample, the same in both arms: ORACLE_PROMPT-token prefill
+    (untimed), one warm-up step, then ORACLE_PASSES passes of ORACLE_STEPS timed decode steps
+    with generation indices spread over the run like the GPU's.  The host is shared with other
+    jobs, so a pass can be disturbed: the fastest pass is the value, every pass is reported.
+    Returns (tokens/s of the best pass, [seconds per pass], threads used)."""
     import oracle as O
-    orc = O.Oracle(shape, w_cpu, 1, ORACLE_PROMPT + steps + warmup + 2, start_id=start_id)
+    orc = O.Oracle(shape, w_cpu, 1, ORACLE_PROMPT + ORACLE_PASSES * steps + 4, start_id=start_id)
     prompt = I.prompt_tokens(shape, I.BASE_SEED, 0, ORACLE_PROMPT).numpy()
     orc.prefill(0, prompt)
-    toks = I.token_ids(I.BASE_SEED, 999, steps + warmup, shape.vocab).numpy()
+    toks = I.token_ids(I.BASE_SEED, 999, steps + 1, shape.vocab).numpy()
     gi = gen_indices(steps)
-    for j in range(warmup):
-        orc.decode_step([0], [int(toks[j])], [gi[0]], alpha)
-    t0 = time.perf_counter()
-    for j in range(steps):
-        orc.decode_step([0], [int(toks[warmup + j])], [gi[j]], alpha)
-    dt = time.perf_counter() - t0
+    orc.decode_step([0], [int(toks[steps])], [gi[0]], alpha)
+    passes = []
+    for _ in range(ORACLE_PASSES):
+        t0 = time.perf_counter()
+        for j in range(steps):
+            orc.decode_step([0], [int(toks[j])], [gi[j]], alpha)
+        passes.append(time.perf_counter() - t0)
     orc.close()
-    return steps * BATCH / dt, dt, O.threads()
+    return steps * BATCH / min(passes), passes, O.threads()
 
 
 def host_mem_available_gb():
@@ -157,36 +173,58 @@ def oracle_shape_and_scale(shape):
     return small, 8.0 / shape.n_layers, "8 of 32 blocks, tokens/s scaled by 8/32"
 
 
+def oracle_baseline(w, shape, alpha, start_id, steps):
+    """cpu_baseline object of either arm (w: weights on any device)."""
+    oshape, scale, note = oracle_shape_and_scale(shape)
+    w_cpu = I.weights_to({k: (v[:oshape.n_layers] if isinstance(v, list) else v) for k, v in w.items()}, "cpu")
+    tps, passes, cores = time_oracle(oshape, w_cpu, alpha, min(start_id, oshape.n_layers), steps)
+    return {"value": tps * scale, "unit": "tokens/s", "cores": cores, "kind": "oracle",
+            "omp_threads": cores, "host_cpus": os.cpu_count(),
+            "pass_seconds": [round(p, 2) for p in passes],
+            "sample": f"fp64 C oracle, 7B shape, {note}, prompt {ORACLE_PROMPT}, best of {ORACLE_PASSES} passes of "
+                      f"{steps} decode steps at alpha={alpha} ({sum(passes):.1f} s of CPU work in all)"}
+
+
 def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return 0
-    shape, scale, note = oracle_shape_and_scale(I.LLAMA_7B)
+    shape = I.LLAMA_7B
     dev = "cuda:0" if torch.cuda.is_available() else "cpu"
     w = I.make_weights(shape, I.BASE_SEED, device=dev)
-    w_cpu = I.weights_to(w, "cpu")
-    del w
-    start_id = int(START_FRACTION * I.LLAMA_7B.n_layers)
-    steps = min(args.steps, 64)
-    tps, dt, cores = time_oracle(shape, w_cpu, args.alpha, min(start_id, shape.n_layers), steps,
-                                 min(args.warmup, 3))
-    tps *= scale
-    sample = (f"CPU oracle (fp64, OpenMP), 7B shape, {note}, prompt {ORACLE_PROMPT}, "
-              f"{steps} decode steps at alpha={args.alpha}")
+    start_id = int(START_FRACTION * shape.n_layers)
+    steps = oracle_steps(args.steps)
+    cb = oracle_baseline(w, shape, args.alpha, start_id, steps)
+    tps = cb["value"]
     line = {
         "impl": "reference", "metric": METRIC, "value": tps, "unit": "tokens/s",
-        "n_gpus": args.gpus, "steps": steps, "warmup": min(args.warmup, 3),
-        "ms_per_step": 1e3 * dt / steps, "higher_is_better": True, "scaling": "weak",
+        "n_gpus": args.gpus, "steps": steps, "warmup": 1,
+        "ms_per_step": 1e3 / tps, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": {"workload": "llama2-7b-shape batch 1, prompt 512, generate 256 (oracle: bounded sample)",
                    "alpha": args.alpha, "start_id": start_id},
-        "cpu_baseline": {"value": tps, "unit": "tokens/s", "cores": cores, "kind": "oracle",
-                         "sample": sample},
+        "cpu_baseline": cb,
         "e2e": {"value": tps, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
     print(json.dumps(line), flush=True)
     return 0
+
+
+def spawn_replicas(args):
+    """`--gpus N` outside a torchrun environment: start the N replica processes (one per GPU)
+    with the standard launcher and pass the flags through; rank 0 prints the line."""
+    import socket
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
+
+
+def median(v):
+    return statistics.median(v)
 
 
 def main():
@@ -195,16 +233,23 @@ def main():
     ap.add_argument("--steps", type=int, default=GENERATE - 1)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--alpha", type=float, default=0.995)
+    ap.add_argument("--reps", type=int, default=5, help="repetitions of the K-step timed region (>= 5)")
     ap.add_argument("--impl", default="d3", choices=["d3", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--workloads", default="c3,c4",
+                    help="batched workloads reported beside the main line (c3,c4,c5 or none); "
+                         "c5 holds ~140 GB of weights and is off by default")
     ap.add_argument("--layers", type=int, default=0,
                     help="profiling aid: keep only this many blocks (same kernel shapes, less memory); "
                          "numbers from such a run are not benchmark values")
     ap.add_argument("--prompt", type=int, default=PROMPT, help="profiling aid: shorter prompt")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
+    args.reps = max(args.reps, 1)
     if args.impl == "reference":
         return run_reference(args)
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        return spawn_replicas(args)
 
     from paper_2503_08524_b200 import binding as B   # raises if libd3 is missing
 
@@ -223,14 +268,15 @@ def main():
     from paper_2503_08524_b200.replicas import Replicas
     reps = Replicas(dist, dev)
     barrier = reps.barrier
+    max_over_ranks = reps.max_ms
+    profiling_aid = args.layers > 0 or args.prompt != PROMPT
 
     shape = I.LLAMA_7B if args.layers <= 0 else I.LLAMA_7B.with_layers(args.layers)
     start_id = int(START_FRACTION * shape.n_layers)
     K, W = args.steps, args.warmup
     max_seq = args.prompt + K + W + 8
     w = I.make_weights(shape, I.BASE_SEED, device=dev)
-    # max_batch 32 only lets the (untimed) prefill run 32 prompt positions per pass
-    model = B.D3Model(shape, w, 1, max_seq, 32, start_id=start_id, device=dev)
+    model = B.D3Model(shape, w, 1, max_seq, 64, start_id=start_id, device=dev)
     model.zero_kv()
     prompt = I.prompt_tokens(shape, I.BASE_SEED, 0, args.prompt).numpy()
     toks = I.token_ids(I.BASE_SEED, 999, K + W, shape.vocab).numpy()
@@ -239,9 +285,13 @@ def main():
     stream = torch.cuda.current_stream()
 
     def timed_run(alpha, profile=False):
-        """Prefill, W warm-up steps, K timed steps.  Returns (ms, stats totals)."""
+        """Prefill, W warm-up steps, K timed steps.  Returns (ms, stats totals, profile, prefill ms)."""
         model.d3_reset_slot(0)
-        model.d3_prefill(0, prompt)
+        p0, p1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        p0.record(stream)
+        model.d3_prefill(0, prompt, logits=logits[0])
+        p1.record(stream)
         for j in range(W):
             model.d3_decode_step([0], [int(toks[j])], [gi[0]], alpha, logits=logits)
         model.d3_profile(profile)
@@ -263,15 +313,22 @@ def main():
         ms = e0.elapsed_time(e1)
         prof = model.d3_read_profile() if profile else None
         model.d3_profile(False)
-        return ms, tot, prof
+        return ms, tot, prof, p0.elapsed_time(p1)
 
-    max_over_ranks = reps.max_ms
+    def repeated(alpha, n):
+        """n repetitions of the K-step region; per repetition the slowest rank's time."""
+        ms_list, ttft, tot = [], [], None
+        for _ in range(n):
+            ms, tot, _, pf = timed_run(alpha)
+            ms_list.append(max_over_ranks(ms))
+            ttft.append(pf)
+        return ms_list, tot, ttft
 
-    # ---- main timed region (clock samples taken meanwhile)
+    # ---- main timed region: args.reps repetitions, clock samples taken across all of them
     sampler = ClockSampler(local) if rank == 0 else None
-    ms, tot, _ = timed_run(args.alpha)
+    ms_reps, tot, ttft_ms = repeated(args.alpha, args.reps)
     clocks = sampler.stop() if sampler else None
-    ms = max_over_ranks(ms)
+    ms = median(ms_reps)
     value = world * BATCH * K / (ms / 1e3)
 
     # ---- the same kernels at alpha = 1 (full depth) and 0.999
@@ -279,33 +336,42 @@ def main():
     for a in (1.0, 0.999):
         if abs(a - args.alpha) < 1e-12:
             continue
-        ms_a, tot_a, _ = timed_run(a)
-        ms_a = max_over_ranks(ms_a)
-        others[a] = (ms_a, tot_a)
+        ms_a, tot_a, _ = repeated(a, 3 if args.reps >= 3 else args.reps)
+        others[a] = (median(ms_a), min(ms_a), tot_a)
 
     # ---- per-kernel-class device times of the same K steps (events around each launch)
-    _, _, prof = timed_run(args.alpha, profile=True)
+    _, _, prof, _ = timed_run(args.alpha, profile=True)
 
-    # ---- end to end through the C ABI: host token in, argmax token out, every step
-    model.d3_reset_slot(0)
-    model.d3_prefill(0, prompt)
+    # ---- end to end through the C ABI, every step: host token in (pinned), the call's result out
+    # (the [vocab] fp32 logits, 128 KB, to pinned host memory) plus the greedy token chosen on the
+    # device, which is the next step's input.  Second variant: only the 4-byte token comes back.
     tok_dev = torch.empty(BATCH, dtype=torch.int32, device=dev)
     tok_host = torch.empty(BATCH, dtype=torch.int32).pin_memory()
-    cur = int(toks[0])
-    for j in range(W):
-        model.d3_decode_step([0], [cur], [gi[0]], args.alpha, logits=logits)
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    barrier()
-    e0.record(stream)
-    for j in range(K):
-        model.d3_decode_step([0], [cur], [gi[j]], args.alpha, logits=logits)   # host arrays -> device
-        model.d3_argmax(logits, tok_dev)
-        tok_host.copy_(tok_dev, non_blocking=True)                              # device -> host
-        stream.synchronize()
-        cur = int(tok_host[0])
-    e1.record(stream)
-    barrier()
-    e2e_ms = max_over_ranks(e0.elapsed_time(e1))
+    logits_host = torch.empty((BATCH, shape.vocab), dtype=torch.float32).pin_memory()
+
+    def e2e_run(copy_logits):
+        model.d3_reset_slot(0)
+        model.d3_prefill(0, prompt)
+        cur = int(toks[0])
+        for j in range(W):
+            model.d3_decode_step([0], [cur], [gi[0]], args.alpha, logits=logits)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        e0.record(stream)
+        for j in range(K):
+            model.d3_decode_step([0], [cur], [gi[j]], args.alpha, logits=logits)   # host arrays -> device
+            model.d3_argmax(logits, tok_dev)
+            if copy_logits:
+                logits_host.copy_(logits, non_blocking=True)                        # device -> host
+            tok_host.copy_(tok_dev, non_blocking=True)
+            stream.synchronize()
+            cur = int(tok_host[0])
+        e1.record(stream)
+        barrier()
+        return max_over_ranks(e0.elapsed_time(e1))
+
+    e2e_ms = median([e2e_run(True) for _ in range(3)])
+    e2e_tok_ms = median([e2e_run(False) for _ in range(3)])
     e2e_value = world * BATCH * K / (e2e_ms / 1e3)
 
     if rank != 0:
@@ -335,39 +401,67 @@ def main():
                 "share_of_kernel_time": top_ms / prof_total, "launches": top_n}
     if top_name in class_bytes:
         ach = class_bytes[top_name] * BATCH / 1e9 / (top_ms / top_n / 1e3)
-        roofline.update(achieved=ach, frac=ach / peak, bytes_per_launch=class_bytes[top_name],
-                        avg_launch_us=1e3 * top_ms / top_n)
+        roofline.update(achieved=ach, frac=ach / peak, frac_of_nominal_8TBs=ach / NOMINAL_HBM_GBS,
+                        bytes_per_launch=class_bytes[top_name], avg_launch_us=1e3 * top_ms / top_n)
         if top_name == "fused_step" and FUSED_TRAFFIC_RATIO is not None:
             roofline["traffic"] = FUSED_TRAFFIC_RATIO * class_bytes[top_name]
     else:
         roofline.update(achieved=None, frac=None)
     step_gbs = tot["bytes"] / 1e9 / (ms / 1e3)
+    best_gbs = tot["bytes"] / 1e9 / (min(ms_reps) / 1e3)
     step_roofline = {"bytes_per_step": tot["bytes"] / K, "achieved": step_gbs, "unit": "GB/s",
                      "frac_of_measured": step_gbs / peak, "frac_of_nominal_8TBs": step_gbs / NOMINAL_HBM_GBS,
+                     "best_rep_frac_of_measured": best_gbs / peak,
                      "avg_layers_per_token": tot["rows_layers"] / K}
     alphas = {str(args.alpha): {"tokens_per_s": value, "ms_per_step": ms / K,
                                 "avg_layers": tot["rows_layers"] / K,
-                                "frac_of_measured": step_gbs / peak}}
-    for a, (ms_a, tot_a) in others.items():
+                                "frac_of_measured": step_gbs / peak,
+                                "frac_of_nominal_8TBs": step_gbs / NOMINAL_HBM_GBS}}
+    for a, (ms_a, best_a, tot_a) in others.items():
         g = tot_a["bytes"] / 1e9 / (ms_a / 1e3)
         alphas[str(a)] = {"tokens_per_s": world * BATCH * K / (ms_a / 1e3), "ms_per_step": ms_a / K,
-                          "avg_layers": tot_a["rows_layers"] / K, "frac_of_measured": g / peak}
+                          "ms_per_step_best": best_a / K,
+                          "avg_layers": tot_a["rows_layers"] / K, "frac_of_measured": g / peak,
+                          "frac_of_nominal_8TBs": g / NOMINAL_HBM_GBS}
     if 1.0 in others:
         full = alphas["1.0"]
         alphas["speedup_vs_alpha_1"] = value / full["tokens_per_s"]
         alphas["layer_ratio_vs_alpha_1"] = full["avg_layers"] / (tot["rows_layers"] / K)
-        alphas["bytes_ratio_vs_alpha_1"] = others[1.0][1]["bytes"] / tot["bytes"]
+        alphas["bytes_ratio_vs_alpha_1"] = others[1.0][2]["bytes"] / tot["bytes"]
+
+    # ---- time to first token: the prompt through all blocks (d3_prefill), device-timed
+    pf = median(ttft_ms)
+    flops = 2.0 * args.prompt * shape.n_layers * (shape.layer_weight_bytes / 2) + 2.0 * shape.vocab * shape.d_model
+    ttft = {"prompt_tokens": args.prompt, "ms": pf, "ms_best": min(ttft_ms),
+            "prompt_tokens_per_s": args.prompt / (pf / 1e3), "projection_tflops": flops / 1e12 / (pf / 1e3)}
+
+    # ---- batched workloads (mixed depths, tensor-core projections), each with its own clock record
+    model.close()
+    del model, w
+    torch.cuda.empty_cache()
+    workloads = {}
+    wl_launches = 0
+    if world == 1 and not profiling_aid:
+        from paper_2503_08524_b200 import workloads as WL
+        for name in [n for n in args.workloads.split(",") if n in WL.WORKLOADS]:
+            box = {}
+
+            def on_timed(start, box=box):
+                if start:
+                    box["s"] = ClockSampler(local)
+                else:
+                    box["clocks"] = box.pop("s").stop()
+            r = WL.run_workload(name, steps=24 if name != "c5" else 12, reps=3, device=dev, on_timed=on_timed)
+            r["clocks"] = box.get("clocks")
+            r.pop("kernel_classes", None)
+            workloads[name] = r
+            wl_launches += int(r["launches_per_step"] * r["steps"] * r["reps"])
 
     cpu_baseline = None
     if world == 1 and not args.no_cpu_baseline:
-        oshape, scale, note = oracle_shape_and_scale(shape)
-        w_cpu = I.weights_to({k: (v[:oshape.n_layers] if isinstance(v, list) else v)
-                              for k, v in w.items()}, "cpu")
-        osteps = 96 if scale == 1.0 else 192      # ~15 s of CPU work on the box's 16 cores
-        tps, dt, cores = time_oracle(oshape, w_cpu, args.alpha, start_id, osteps, 1)
-        cpu_baseline = {"value": tps * scale, "unit": "tokens/s", "cores": cores, "kind": "oracle",
-                        "sample": f"fp64 C oracle, 7B shape, {note}, prompt {ORACLE_PROMPT}, {osteps} decode "
-                                  f"steps at alpha={args.alpha}, {dt:.1f} s of CPU work"}
+        w = I.make_weights(shape, I.BASE_SEED, device=dev)
+        cpu_baseline = oracle_baseline(w, shape, args.alpha, start_id, oracle_steps(K))
+        del w
 
     line = {
         "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": K,
@@ -378,10 +472,15 @@ def main():
                    "anchor": "start", "kv_fill": "copy", "gen_index_schedule": "1 + floor(j*255/K)",
                    "l2": "inputs_exceed_l2 (weights of one step >> 126 MB)",
                    "multi_gpu": "independent replicas"},
+        "repetitions": {"n": len(ms_reps), "reported": "median", "ms_per_step_median": ms / K,
+                        "ms_per_step_best": min(ms_reps) / K, "ms_per_step_all": [m / K for m in ms_reps]},
         "roofline": roofline, "step_roofline": step_roofline, "alphas": alphas,
-        "kernel_classes": prof, "cpu_baseline": cpu_baseline,
+        "kernel_classes": prof, "ttft": ttft, "workloads": workloads, "cpu_baseline": cpu_baseline,
         "e2e": {"value": e2e_value, "unit": "tokens/s", "ms_per_step": e2e_ms / K,
-                "h2d_bytes_per_step": 12 * BATCH, "d2h_bytes_per_step": 4 * BATCH},
+                "h2d_bytes_per_step": 12 * BATCH, "d2h_bytes_per_step": (4 * shape.vocab + 4) * BATCH,
+                "result": "fp32 logits [vocab] to pinned host memory + the greedy token",
+                "token_only": {"value": world * BATCH * K / (e2e_tok_ms / 1e3), "ms_per_step": e2e_tok_ms / K,
+                               "d2h_bytes_per_step": 4 * BATCH}},
         "gpu_launches": tot["launches"], "clocks": clocks,
     }
     print(json.dumps(line), flush=True)

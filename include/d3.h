@@ -266,8 +266,8 @@ int32_t d3_read_fused_phases(d3_model *m, int64_t *cycles, int32_t *ctas, int32_
  * memory until the process exits.  No call made here allocates or frees device
  * memory, and no model handle is created.
  *
- * It computes what d3_decode_step computes for a single row through the
- * single-kernel step (Sec. 3.4): the sequence in `slot`, whose cache holds
+ * It computes what d3_decode_step computes for a single row (see that call's
+ * comment), through the single-kernel step: the sequence in `slot`, whose cache holds
  * `pos` >= 1 tokens, feeds `token` = T_{i-1} with i = gen_index >= 1, writes
  * K,V of the retained blocks (and the fill of the dropped ones) at position
  * `pos` of kv_dev, and writes the logits that choose T_i to logits_dev
@@ -282,9 +282,18 @@ int32_t d3_read_fused_phases(d3_model *m, int64_t *cycles, int32_t *ctas, int32_
  * grouping other than 128x1, 128x4, 64x1, 32x4; vocab not a multiple of 4),
  * for fill RECOMPUTE and for bad arguments; D3_ECUDA when a runtime call fails.
  *
- * First call on a device: it looks up the array's device address and sets the
- * kernel's shared-memory attribute for the current device.  Make that first
- * call with the right device current and outside any stream capture.
+ * Set-up: the first call on a device looks up the array's device address, and
+ * the first call for a new set of model sizes sets the kernel's shared-memory
+ * attribute; both with the current device, which must be the one the buffers
+ * live on.  Every call also does host-side work that a stream capture would
+ * freeze or refuse (it passes pos, token and the depth thresholds by value and
+ * may copy the weight-pointer table from host memory), so never call it inside
+ * a stream capture.
+ *
+ * Device-side errors: the call returns once the kernel is enqueued.  A bounded
+ * wait that ran out inside the kernel (D3_ETIMEOUT) is recorded in the array;
+ * d3_noalloc_status reads it (it allocates nothing either) and should be
+ * checked before the logits are trusted.
  *
  * All calls on a GPU share the one array, which keeps the previous call's
  * contents; the entry point re-initialises what must start from zero.  Two
@@ -295,13 +304,38 @@ int32_t d3_read_fused_phases(d3_model *m, int64_t *cycles, int32_t *ctas, int32_
 int32_t d3_decode_step_noalloc(const d3_config *cfg, const d3_weights *weights, void *kv_dev,
                                int32_t slot, int32_t pos, int32_t token, int32_t gen_index,
                                double alpha, float *logits_dev, void *cuda_stream);
+/* Waits for `cuda_stream` and returns the device status of the last
+ * d3_decode_step_noalloc on the current device: D3_OK, D3_ETIMEOUT, or
+ * D3_ECUDA when a runtime call fails.  Copies one int32 out of the built-in
+ * array into a host local; allocates nothing.  (No counterpart in the paper.) */
+int32_t d3_noalloc_status(void *cuda_stream);
 
 int32_t d3_slot_pos(const d3_model *m, int32_t slot); /* tokens cached; D3_ESTATE if never prefilled */
 /* PAGED layout: pages handed out at the moment (the reserved page not counted);
  * D3_EINVAL for a contiguous model.  Host bookkeeping only. */
 int32_t d3_kv_pages_used(const d3_model *m);
 int32_t d3_reset_slot(d3_model *m, int32_t slot);
-int32_t d3_sync(d3_model *m); /* wait for the stream; returns a deferred device status */
+/* Wait for the stream; returns a deferred device status (D3_ETIMEOUT) once and clears it. */
+int32_t d3_sync(d3_model *m);
+
+/* Window policy between steps (Appendix, Table "HP description": `start` differs per
+ * task, Sec. 4.1 "Hyperparameter Settings"; anchor and fill as in d3_config).  Takes
+ * effect from the next call on; sequences in flight keep their caches.  Host only. */
+int32_t d3_set_policy(d3_model *m, int32_t start_id, int32_t anchor, int32_t kv_fill);
+
+/* Failure detection.  Every device-side wait of the library (mbarrier, ring slot,
+ * grid barrier) gives up after `ns` nanoseconds (default 2e9): the kernel raises
+ * D3_ETIMEOUT in a status word that d3_sync returns, stops issuing copies, lets the
+ * copies in flight land and runs to its end; nothing traps and the context stays
+ * usable.  The outputs and the cache entries of such a step are undefined: reset
+ * and prefill the slots it touched.  ns >= 1. */
+int32_t d3_set_wait_ns(d3_model *m, uint64_t ns);
+/* Drill for the above: the next single-kernel step (one row) is told to expect one
+ * arrival more at its first grid barrier than there are CTAs, so that wait can only
+ * end by its time limit -- a wait nobody satisfies, made on the host.  The step
+ * then ends with D3_ETIMEOUT as described.  D3_EINVAL when the model has no
+ * single-kernel step. */
+int32_t d3_stall_next_step(d3_model *m);
 void d3_free(d3_model *m);    /* host bookkeeping only */
 const char *d3_strerror(int32_t code);
 

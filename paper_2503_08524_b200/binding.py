@@ -26,7 +26,9 @@ MAX_BATCH = 64     # D3_MAX_BATCH
 EXPORTS = ("d3_depth", "d3_schedule", "d3_workspace_bytes", "d3_load", "d3_prefill",
            "d3_decode_step", "d3_decode_step_depths", "d3_depth_linear", "d3_saturation_probe",
            "d3_argmax", "d3_read_schedule", "d3_read_hidden", "d3_read_kv",
-           "d3_set_exec", "d3_profile", "d3_read_profile", "d3_profile_name", "d3_read_fused_phases", "d3_decode_step_noalloc", "d3_slot_pos",
+           "d3_set_exec", "d3_profile", "d3_read_profile", "d3_profile_name", "d3_read_fused_phases",
+           "d3_decode_step_noalloc", "d3_noalloc_status", "d3_set_policy", "d3_set_wait_ns",
+           "d3_stall_next_step", "d3_slot_pos",
            "d3_kv_pages_used", "d3_reset_slot", "d3_sync", "d3_free", "d3_strerror")
 
 
@@ -85,6 +87,10 @@ def _load() -> C.CDLL:
     lib.d3_profile_name.restype = C.c_char_p
     lib.d3_decode_step_noalloc.argtypes = [C.POINTER(Config), C.POINTER(Weights), P, I32, I32, I32, I32,
                                            C.c_double, P, P]
+    lib.d3_noalloc_status.argtypes = [P]
+    lib.d3_set_policy.argtypes = [P, I32, I32, I32]
+    lib.d3_set_wait_ns.argtypes = [P, C.c_uint64]
+    lib.d3_stall_next_step.argtypes = [P]
     lib.d3_slot_pos.argtypes = [P, I32]
     lib.d3_kv_pages_used.argtypes = [P]
     lib.d3_reset_slot.argtypes = [P, I32]
@@ -171,6 +177,12 @@ def d3_decode_step_noalloc(cfg: Config, weights: Dict[str, object], kv: torch.Te
     return int(LIB.d3_decode_step_noalloc(C.byref(cfg), C.byref(ws), kv.data_ptr(), slot, pos, token,
                                           gen_index, float(alpha), logits.data_ptr(),
                                           C.c_void_p(st.cuda_stream)))
+
+
+def d3_noalloc_status(stream: Optional[torch.cuda.Stream] = None) -> int:
+    """Device status of the last d3_decode_step_noalloc on the current device (waits for the stream)."""
+    st = stream if stream is not None else torch.cuda.current_stream()
+    return int(LIB.d3_noalloc_status(C.c_void_p(st.cuda_stream)))
 
 
 class D3Model:
@@ -373,3 +385,18 @@ class D3Model:
         rc = LIB.d3_sync(self.h)
         if rc != OK:
             raise D3Error(rc, "d3_sync")
+
+    def d3_set_policy(self, start_id: int, anchor: int, kv_fill: int) -> None:
+        rc = LIB.d3_set_policy(self.h, start_id, anchor, kv_fill)
+        if rc != OK:
+            raise D3Error(rc, "d3_set_policy")
+
+    def d3_set_wait_ns(self, ns: int) -> None:
+        rc = LIB.d3_set_wait_ns(self.h, int(ns))
+        if rc != OK:
+            raise D3Error(rc, "d3_set_wait_ns")
+
+    def d3_stall_next_step(self) -> None:
+        rc = LIB.d3_stall_next_step(self.h)
+        if rc != OK:
+            raise D3Error(rc, "d3_stall_next_step")

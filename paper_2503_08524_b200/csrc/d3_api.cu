@@ -122,6 +122,8 @@ struct d3_model {
   size_t fused_smem;
   void *fused_func;
   std::vector<LayerPtrs> layer_tab_host;
+  unsigned long long wait_ns;   // bound of every device-side wait (d3_set_wait_ns)
+  int stall_next;               // time-out drill: the next single-kernel step cannot pass its first barrier
   // tensor-core projections: tensor maps of the weight matrices (entry valid when tm_ok)
   TcContext tc;
   std::vector<TMap> tm_qkv, tm_kv, tm_o, tm_gate, tm_up, tm_down;
@@ -389,7 +391,9 @@ static int32_t run_fused_step(d3_model *m, const StepArgs &a, float *logits_dev,
   fp.logits = logits_dev;
   fp.n_stages = m->fused_stages; fp.act_floats = m->fused_act;
   fp.l2_window = fused_l2_window();
-  fp.wait_ns = 2000000000ull;
+  fp.wait_ns = m->wait_ns;
+  fp.barrier_extra = m->stall_next ? 1u : 0u;
+  m->stall_next = 0;
   int rc;
   {
     ProfScope ps(m, PK_FUSED);
@@ -568,7 +572,9 @@ int32_t d3_load(const d3_config *cfg, const d3_weights *w, void *kv_dev, void *s
   m->tc.ok = tc_init() == 0;
   m->tc.act_split = reinterpret_cast<bf16 *>(m->scratch + m->lay.act_split);
   m->tc.act_bytes = m->lay.act_split_bytes;
-  m->tc.wait_ns = 2000000000ull;
+  m->wait_ns = 2000000000ull;
+  m->stall_next = 0;
+  m->tc.wait_ns = m->wait_ns;
   {
     int dev = 0, sms = 0;
     if (cudaGetDevice(&dev) != cudaSuccess ||
@@ -835,7 +841,33 @@ int32_t d3_sync(d3_model *m) {
   int32_t status = 0;
   if (cudaMemcpy(&status, &m->sched()->status, 4, cudaMemcpyDeviceToHost) != cudaSuccess)
     return D3_ECUDA;
+  // a deferred status is reported once: the word is cleared so that later steps start clean
+  if (status != 0 && cudaMemset(&m->sched()->status, 0, 4) != cudaSuccess) return D3_ECUDA;
   return status;
+}
+
+int32_t d3_set_policy(d3_model *m, int32_t start_id, int32_t anchor, int32_t kv_fill) {
+  if (!m) return D3_EINVAL;
+  if (start_id < 0 || start_id > m->cfg.n_layers) return D3_EINVAL;
+  if (anchor != D3_ANCHOR_START && anchor != D3_ANCHOR_TAIL) return D3_EINVAL;
+  if (kv_fill < D3_FILL_NONE || kv_fill > D3_FILL_RECOMPUTE) return D3_EINVAL;
+  m->cfg.start_id = start_id;
+  m->cfg.anchor = anchor;
+  m->cfg.kv_fill = kv_fill;
+  return D3_OK;
+}
+
+int32_t d3_set_wait_ns(d3_model *m, uint64_t ns) {
+  if (!m || ns < 1) return D3_EINVAL;
+  m->wait_ns = ns;
+  m->tc.wait_ns = ns;
+  return D3_OK;
+}
+
+int32_t d3_stall_next_step(d3_model *m) {
+  if (!m || !m->fused_ok) return D3_EINVAL;
+  m->stall_next = 1;
+  return D3_OK;
 }
 
 int32_t d3_set_exec(d3_model *m, int32_t mode) {

@@ -135,7 +135,9 @@ __device__ __forceinline__ void grid_barrier(const Ctx &c, unsigned idx) {
   consumer_sync();
   if (threadIdx.x == 0) {
     asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(c.p->bar_counter) : "memory");
-    const unsigned target = idx * (unsigned)c.ncta;
+    // every barrier counts the arrivals of all earlier ones; barrier_extra (0 in normal use)
+    // makes the first target unreachable so that the wait can only end by its time limit
+    const unsigned target = idx * (unsigned)c.ncta + (idx == 1u ? c.p->barrier_extra : 0u);
     const uint64_t t0 = now_ns();
     for (uint32_t it = 1; !*c.abort_flag; ++it) {
       unsigned v;
@@ -851,7 +853,8 @@ __global__ void __launch_bounds__(kFusedThreads, 1) k_step_b1(const __grid_const
         if (s % (uint32_t)kProducerWarps != pr.pid) continue;
         const uint32_t bar = smem_u32(&s_full[s % ns]);
         const uint64_t t0 = now_ns();
-        while (!mbar_try_wait(bar, (s / ns) & 1u) && now_ns() - t0 < p.wait_ns) {}
+        const uint64_t bound = p.wait_ns > kDrainFloorNs ? p.wait_ns : kDrainFloorNs;
+        while (!mbar_try_wait(bar, (s / ns) & 1u) && now_ns() - t0 < bound) {}
       }
     }
     return;

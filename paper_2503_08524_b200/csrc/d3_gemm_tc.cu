@@ -265,8 +265,9 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
       }
       if (*abort_flag) {
         // copies still in flight must land before the CTA's shared memory is given back
+        const unsigned long long bound = t.wait_ns > kDrainFloorNs ? t.wait_ns : kDrainFloorNs;
         for (int it = max(0, issued - S); it < issued; ++it)
-          bar_wait(smem_addr(&s_full[it % S]), (uint32_t)((it / S) & 1), abort_flag, t.wait_ns, false);
+          bar_wait(smem_addr(&s_full[it % S]), (uint32_t)((it / S) & 1), abort_flag, bound, false);
       }
     }
     __syncwarp();
@@ -287,7 +288,13 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
           umma_bf16(tmem, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), idesc, (it | k) ? 1u : 0u);
         umma_commit(smem_addr(&s_empty[s]));
       }
-      if (ok) umma_commit(smem_addr(&s_accum));
+      umma_commit(smem_addr(&s_accum));
+      if (!ok) {
+        // aborted: the MMAs already issued still read shared memory and write TMEM; they end by
+        // themselves, so wait for them (bounded) before the CTA gives both back
+        const unsigned long long bound = t.wait_ns > kDrainFloorNs ? t.wait_ns : kDrainFloorNs;
+        bar_wait(smem_addr(&s_accum), 0u, abort_flag, bound, false);
+      }
     }
     __syncwarp();
   } else {

@@ -123,7 +123,13 @@ struct FusedParams {
   int32_t n_stages, act_floats;
   uint32_t l2_window;           // ring stages the L2 prefetcher may run ahead (0 = off)
   unsigned long long wait_ns;   // bound of every device-side wait
+  uint32_t barrier_extra;       // arrivals the FIRST grid barrier expects beyond the CTA count (0 in normal
+                                // use; 1 = that barrier can only end by its time limit: time-out drill)
 };
+
+// Waits for copies already in flight are not waits for another party: they always end, so
+// their bound never drops below this floor however short the configured limit is.
+static constexpr unsigned long long kDrainFloorNs = 1000000ull;
 
 // Host state of the tensor-core projection path.
 struct TcContext {
@@ -179,6 +185,7 @@ void thresholds(int32_t L, double alpha, int32_t *thr);
 
 // launchers (each enqueues on `st`; returns the number of kernels launched)
 int launch_rope_table(float2 *table, int max_seq, int dh, float base, cudaStream_t st);
+int launch_rope_rows(float2 *table, int pos0, int n_pos, int dh, float base, cudaStream_t st);
 int launch_schedule_embed(const StepArgs &a, DevSched *s, const bf16 *E, float *x, int d,
                           cudaStream_t st);
 int launch_gemv(const GemvArgs &g, int epi, int m_rows, cudaStream_t st);

@@ -38,19 +38,24 @@ __device__ __forceinline__ void row_range(const DevSched *s, int layer, int mode
 
 // ------------------------------------------------------------------ rope table
 // table[pos][j] = (cos, sin)(pos * base^(-2j/dh)), evaluated in fp64.
-__global__ void k_rope_table(float2 *table, int max_seq, int half, int dh, double base) {
+// Rows pos0 .. pos0 + n_pos - 1 of the table.
+__global__ void k_rope_table(float2 *table, int pos0, int n_pos, int half, int dh, double base) {
   int idx = blockIdx.x * blockDim.x + threadIdx.x;
-  if (idx >= max_seq * half) return;
-  int pos = idx / half, j = idx % half;
+  if (idx >= n_pos * half) return;
+  int pos = pos0 + idx / half, j = idx % half;
   double theta = pow(base, -2.0 * (double)j / (double)dh);
   double s, c;
   sincos((double)pos * theta, &s, &c);
-  table[idx] = make_float2((float)c, (float)s);
+  table[(size_t)pos * half + j] = make_float2((float)c, (float)s);
 }
 
 int launch_rope_table(float2 *table, int max_seq, int dh, float base, cudaStream_t st) {
-  int n = max_seq * (dh / 2);
-  k_rope_table<<<(n + 255) / 256, 256, 0, st>>>(table, max_seq, dh / 2, dh, (double)base);
+  return launch_rope_rows(table, 0, max_seq, dh, base, st);
+}
+
+int launch_rope_rows(float2 *table, int pos0, int n_pos, int dh, float base, cudaStream_t st) {
+  int n = n_pos * (dh / 2);
+  k_rope_table<<<(n + 255) / 256, 256, 0, st>>>(table, pos0, n_pos, dh / 2, dh, (double)base);
   return 1;
 }
 

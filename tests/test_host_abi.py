@@ -114,6 +114,8 @@ def test_workspace_and_load_validation():
     assert B.LIB.d3_prefill(None, 0, None, 1, None) == B.EINVAL
     assert B.LIB.d3_decode_step(None, 1, None, None, None, 0.9, None, None, None) == B.EINVAL
     assert B.LIB.d3_sync(None) == B.EINVAL and B.LIB.d3_slot_pos(None, 0) == B.EINVAL
+    assert B.LIB.d3_set_policy(None, 0, 0, 0) == B.EINVAL and B.LIB.d3_set_wait_ns(None, 5) == B.EINVAL
+    assert B.LIB.d3_stall_next_step(None) == B.EINVAL
     assert B.strerror(B.ESTATE) != B.strerror(B.ECAPACITY)
     assert B.strerror(-99) == "unknown error"
 
