@@ -49,7 +49,7 @@ ORACLE_PROMPT = 32            # bounded sample for the CPU oracle
 # ncu capture summarised in profiles/fused_step_k_step_b1_7bshape_L4.md (4-block case of the same
 # kernel: 1.8917 GB moved for 1.881 GB algorithmic; traffic grows with the blocks executed, so the
 # full launch is scaled by its own algorithmic bytes).  Set to None when the kernel changes.
-FUSED_TRAFFIC_RATIO = 1.0057
+FUSED_TRAFFIC_RATIO = None
 
 
 def gen_indices(k: int):

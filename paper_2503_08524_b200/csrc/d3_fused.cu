@@ -211,6 +211,13 @@ __device__ __forceinline__ const bf16 *group_row(const Phase &ph, const Dims &dm
 // (s*P + k) mod #CTAs.  A part may be empty; it still writes an (empty) partial.
 struct AttPlan {
   int CH, nch, streams, P, parts, gq;
+  // partials in the scratch buffer: o[part][gq][dh] (unnormalised), then (max, sum)[part][gq]
+  __device__ __forceinline__ float *part_o(float *base, int part, int dh) const {
+    return base + (size_t)part * (gq * dh);
+  }
+  __device__ __forceinline__ float *part_ml(float *base, int part, int dh) const {
+    return base + (size_t)parts * (gq * dh) + (size_t)part * (gq * 2);
+  }
 };
 
 __device__ __forceinline__ AttPlan make_att(const FusedParams &p, int gq, int ncta) {
@@ -557,9 +564,9 @@ struct Consumer {
     }
   }
 
-  // Attention of this CTA's parts.  Each part yields one partial (max, sum,
-  // unnormalised o) in part[stream * P + k][gq][dh + 2]; the partials are merged
-  // by merge_load_attn after the grid barrier.
+  // Attention of this CTA's parts.  Each part yields one partial: unnormalised o
+  // [gq][dh] and (max, sum) [gq] of part stream * P + k; the partials are merged by
+  // merge_load_attn after the grid barrier.
   template <int DH, int GQ>
   __device__ void att_phase(const AttPlan &a, int layer) {
     const FusedParams &p = *c.p;
@@ -578,12 +585,11 @@ struct Consumer {
       const int kvh = stream / qgroups, qg = stream % qgroups;
       const int h0 = kvh * G + qg * GQ;
       const int ch0 = a.nch * kpart / a.P, ch1 = a.nch * (kpart + 1) / a.P;
-      float *dst = p.part + (size_t)part * (GQ * (DH + 2));
+      float *dst = a.part_o(p.part, part, DH);
+      float *dst_ml = a.part_ml(p.part, part, DH);
       if (ch0 == ch1) {   // nothing to do: an empty partial (weight 0 in the merge)
-        for (int i = tid; i < GQ * (DH + 2); i += kConsumers) {
-          const int e = i % (DH + 2);
-          dst[i] = (e == DH) ? -INFINITY : 0.f;
-        }
+        for (int i = tid; i < GQ * DH; i += kConsumers) dst[i] = 0.f;
+        if (tid < GQ) { dst_ml[2 * tid] = -INFINITY; dst_ml[2 * tid + 1] = 0.f; }
         continue;
       }
       float q[GQ][EPL], mx[GQ], sum[GQ], o[GQ][EPL];
@@ -591,9 +597,11 @@ struct Consumer {
       for (int g = 0; g < GQ; ++g) {
         mx[g] = -INFINITY; sum[g] = 0.f;
 #pragma unroll
-        for (int e = 0; e < EPL; ++e) {
-          q[g][e] = __ldcg(p.qkv + (h0 + g) * DH + part8 * EPL + e) * scale;
-          o[g][e] = 0.f;
+        for (int e = 0; e < EPL; e += 4) {
+          const float4 qv = ldcg4(p.qkv + (h0 + g) * DH + part8 * EPL + e);
+          q[g][e] = qv.x * scale; q[g][e + 1] = qv.y * scale;
+          q[g][e + 2] = qv.z * scale; q[g][e + 3] = qv.w * scale;
+          o[g][e] = o[g][e + 1] = o[g][e + 2] = o[g][e + 3] = 0.f;
         }
       }
       for (int chunk = ch0; chunk < ch1; ++chunk) {
@@ -698,8 +706,8 @@ struct Consumer {
           Ls += s_ml[(w * GQ + g) * 2 + 1] * cf;
           O += s_o[(w * GQ + g) * DH + e] * cf;
         }
-        dst[g * (DH + 2) + e] = O;
-        if (e == 0) { dst[g * (DH + 2) + DH] = M; dst[g * (DH + 2) + DH + 1] = Ls; }
+        dst[g * DH + e] = O;
+        if (e == 0) { dst_ml[2 * g] = M; dst_ml[2 * g + 1] = Ls; }
       }
       consumer_sync();
     }
@@ -707,41 +715,39 @@ struct Consumer {
   }
 
   // act := attention output of all heads, merged from the P partials of every stream
-  // (after the grid barrier).  All loads are issued before the first is used.
+  // (after the grid barrier).  One L2 round trip: the (max, sum) pairs and the first
+  // batch of 16-byte o loads are issued before anything is used; the merge weight
+  // exp(m_k - M) / sum of every (head, part) is computed once, by one thread.
   template <int DH, int GQ>
   __device__ void merge_load_attn(const AttPlan &a, float *s_pm, float *s_pl) {
     const FusedParams &p = *c.p;
     const Dims &dm = p.dm;
     const int tid = threadIdx.x;
-    const int n_out = dm.Hq * DH, P = a.P;
-    // (max, sum) of every (head, part), entry h * kAttParts + k: loaded into registers
-    // here, parked in shared memory only after the first batch of o loads is in flight
+    const int n4 = dm.Hq * DH / 4, P = a.P;
     constexpr int kMl = (kMaxHeads * kAttParts + kConsumers - 1) / kConsumers;
-    float pm_r[kMl], pl_r[kMl];
+    float2 ml_r[kMl];
 #pragma unroll
     for (int q = 0; q < kMl; ++q) {
-      const int idx = q * kConsumers + tid;
-      pm_r[q] = 0.f; pl_r[q] = 0.f;
+      const int idx = q * kConsumers + tid;   // = h * P + k
+      ml_r[q] = make_float2(-INFINITY, 0.f);
       if (idx < dm.Hq * P) {
         const int h = idx / P, k = idx % P;
         // heads are ordered [kv head][query group][g]: stream = h / GQ, g = h % GQ
-        const float *src = p.part + (size_t)((h / GQ) * P + k) * (GQ * (DH + 2)) + (h % GQ) * (DH + 2);
-        pm_r[q] = __ldcg(src + DH);
-        pl_r[q] = __ldcg(src + DH + 1);
+        ml_r[q] = __ldcg(reinterpret_cast<const float2 *>(a.part_ml(p.part, (h / GQ) * P + k, DH)) + (h % GQ));
       }
     }
-    constexpr int kBatch = 16;
-    for (int j0 = 0; j0 * kConsumers < n_out; j0 += kBatch) {
-      float r[kBatch][kAttParts];
+    constexpr int kBatch = 4;   // float4 outputs per thread and batch
+    for (int j0 = 0; j0 * kConsumers < n4; j0 += kBatch) {
+      float4 r[kBatch][kAttParts];
 #pragma unroll
       for (int jj = 0; jj < kBatch; ++jj) {
-        const int i = (j0 + jj) * kConsumers + tid;
+        const int i4 = (j0 + jj) * kConsumers + tid;
 #pragma unroll
         for (int k = 0; k < kAttParts; ++k) {
-          r[jj][k] = 0.f;
-          if (i < n_out && k < P) {
-            const int h = i / DH, e = i % DH;
-            r[jj][k] = __ldcg(p.part + (size_t)((h / GQ) * P + k) * (GQ * (DH + 2)) + (h % GQ) * (DH + 2) + e);
+          r[jj][k] = make_float4(0.f, 0.f, 0.f, 0.f);
+          if (i4 < n4 && k < P) {
+            const int h = (i4 * 4) / DH, e = (i4 * 4) % DH;
+            r[jj][k] = ldcg4(a.part_o(p.part, (h / GQ) * P + k, DH) + (h % GQ) * DH + e);
           }
         }
       }
@@ -750,31 +756,41 @@ struct Consumer {
         for (int q = 0; q < kMl; ++q) {
           const int idx = q * kConsumers + tid;
           if (idx < dm.Hq * P) {
-            s_pm[(idx / P) * kAttParts + idx % P] = pm_r[q];
-            s_pl[(idx / P) * kAttParts + idx % P] = pl_r[q];
+            s_pm[(idx / P) * kAttParts + idx % P] = ml_r[q].x;
+            s_pl[(idx / P) * kAttParts + idx % P] = ml_r[q].y;
           }
         }
         consumer_sync();   // the (max, sum) table is complete
+        if (tid < dm.Hq) {   // merge weights of head tid, in place of its maxima
+          float M = -INFINITY;
+          for (int k = 0; k < P; ++k) M = fmaxf(M, s_pm[tid * kAttParts + k]);
+          float wk[kAttParts], Ls = 0.f;
+#pragma unroll
+          for (int k = 0; k < kAttParts; ++k) {
+            wk[k] = k < P ? __expf(s_pm[tid * kAttParts + k] - M) : 0.f;   // exp(-inf) = 0: an empty part
+            if (k < P) Ls += s_pl[tid * kAttParts + k] * wk[k];
+          }
+          const float inv = 1.f / Ls;
+#pragma unroll
+          for (int k = 0; k < kAttParts; ++k) s_pm[tid * kAttParts + k] = wk[k] * inv;
+        }
+        consumer_sync();
       }
 #pragma unroll
       for (int jj = 0; jj < kBatch; ++jj) {
-        const int i = (j0 + jj) * kConsumers + tid;
-        if (i < n_out) {
-          const int h = i / DH;
-          float M = -INFINITY;
-#pragma unroll
-          for (int k = 0; k < kAttParts; ++k)
-            if (k < P) M = fmaxf(M, s_pm[h * kAttParts + k]);
-          float Ls = 0.f, O = 0.f;
+        const int i4 = (j0 + jj) * kConsumers + tid;
+        if (i4 < n4) {
+          const int h = (i4 * 4) / DH;
+          float4 O = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
           for (int k = 0; k < kAttParts; ++k) {
             if (k < P) {
-              const float cf = __expf(s_pm[h * kAttParts + k] - M);   // exp(-inf) = 0 for an empty part
-              Ls += s_pl[h * kAttParts + k] * cf;
-              O += r[jj][k] * cf;
+              const float wgt = s_pm[h * kAttParts + k];
+              O.x += r[jj][k].x * wgt; O.y += r[jj][k].y * wgt;
+              O.z += r[jj][k].z * wgt; O.w += r[jj][k].w * wgt;
             }
           }
-          c.act[act_index(i)] = O / Ls;
+          *reinterpret_cast<float4 *>(c.act + act_index(i4 * 4)) = O;
         }
       }
     }
