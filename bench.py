@@ -276,7 +276,7 @@ def main():
     K, W = args.steps, args.warmup
     max_seq = args.prompt + K + W + 8
     w = I.make_weights(shape, I.BASE_SEED, device=dev)
-    model = B.D3Model(shape, w, 1, max_seq, 64, start_id=start_id, device=dev)
+    model = B.D3Model(shape, w, 1, max_seq, 128, start_id=start_id, device=dev)
     model.zero_kv()
     prompt = I.prompt_tokens(shape, I.BASE_SEED, 0, args.prompt).numpy()
     toks = I.token_ids(I.BASE_SEED, 999, K + W, shape.vocab).numpy()

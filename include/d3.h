@@ -38,7 +38,7 @@ extern "C" {
 #define D3_ECUDA (-4)     /* a CUDA runtime call failed                                */
 #define D3_ETIMEOUT (-5)  /* a bounded device-side wait ran out                         */
 
-#define D3_MAX_BATCH 64   /* rows per step                                             */
+#define D3_MAX_BATCH 128  /* rows per step (decode rows, or prompt positions per prefill pass) */
 #define D3_MAX_LAYERS 128
 
 /* Which blocks a token with retained count n drops. */
@@ -80,7 +80,9 @@ typedef struct d3_config {
   float rope_base;
   int32_t max_slots;        /* sequences the KV cache holds                            */
   int32_t max_seq;          /* positions per sequence                                  */
-  int32_t max_batch;        /* rows per decode step, 1..D3_MAX_BATCH                   */
+  int32_t max_batch;        /* rows per decode step, 1..D3_MAX_BATCH; also the prompt
+                               positions one prefill pass takes (the weights are streamed
+                               once per pass: 128 gives the shortest time to first token) */
   int32_t start_id;         /* 0..L: first droppable block, 0-based (floor(start * L)) */
   int32_t anchor;           /* D3_ANCHOR_*                                             */
   int32_t kv_fill;          /* D3_FILL_*                                               */
@@ -149,7 +151,10 @@ int32_t d3_load(const d3_config *cfg, const d3_weights *weights, void *kv_dev, v
 /* Initiation phase (Sec. 3.1; Sec. 4.1: prompts pass through all blocks): run
  * every prompt token through all L blocks, fill the slot's cache from position
  * 0, and write the logits that choose T_0 to logits_dev [vocab] (fp32; may be
- * NULL).  Resets the slot first. */
+ * NULL).  Resets the slot first.  The prompt is taken in passes of up to
+ * max_batch consecutive positions: per pass the projections are tensor-core
+ * GEMMs over all its positions (each weight read once per pass) and the
+ * attention is a causal flash-attention kernel over the cache. */
 int32_t d3_prefill(d3_model *m, int32_t slot, const int32_t *tokens, int32_t n_tokens,
                    float *logits_dev);
 

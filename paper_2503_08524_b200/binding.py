@@ -18,10 +18,9 @@ from . import build as _build
 OK, EINVAL, ECAPACITY, ESTATE, ECUDA, ETIMEOUT = 0, -1, -2, -3, -4, -5
 ANCHOR_START, ANCHOR_TAIL = 0, 1
 FILL_NONE, FILL_COPY, FILL_RECOMPUTE = 0, 1, 2
-MAX_BATCH, MAX_LAYERS, PROF_KINDS = 64, 128, 22
+MAX_BATCH, MAX_LAYERS, PROF_KINDS = 128, 128, 22
 EXEC_AUTO, EXEC_KERNELS, EXEC_TENSOR, EXEC_FUSED = 0, 1, 2, 3
 KV_CONTIGUOUS, KV_PAGED = 0, 1
-MAX_BATCH = 64     # D3_MAX_BATCH
 
 EXPORTS = ("d3_depth", "d3_schedule", "d3_workspace_bytes", "d3_load", "d3_prefill",
            "d3_decode_step", "d3_decode_step_depths", "d3_depth_linear", "d3_saturation_probe",

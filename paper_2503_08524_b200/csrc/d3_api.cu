@@ -144,6 +144,9 @@ struct d3_model {
   float *u() const { return reinterpret_cast<float *>(scratch + lay.u); }
 };
 
+// prefill passes of at least this many positions take the causal flash-attention kernel
+static constexpr int kPrefillAttnMinRows = 8;
+
 enum ProfKind { PK_SCHED = 0, PK_QKV, PK_ROPE, PK_ATTN, PK_OPROJ, PK_GATEUP, PK_DOWN, PK_FILL,
                 PK_HEAD, PK_FUSED };
 static const char *kProfNames[D3_PROF_KINDS] = {
@@ -260,7 +263,7 @@ struct ProbeOut {
 static int32_t run_step(d3_model *m, const StepArgs &a, const int32_t *n, const int32_t *lo,
                         const int32_t *hi, const int32_t *perm, const int32_t *m_l,
                         float *logits_dev, int logits_mode, int32_t *launches_out,
-                        const ProbeOut *probe = nullptr) {
+                        const ProbeOut *probe = nullptr, int prefill_t0 = -1) {
   const d3_config &c = m->cfg;
   const Dims &dm = m->dm;
   cudaStream_t st = m->stream;
@@ -294,6 +297,12 @@ static int32_t run_step(d3_model *m, const StepArgs &a, const int32_t *n, const 
         launches += launch_rope_append(m->qkv(), m->rope(), m->Kc, m->Vc, m->sched(), l, ROWS_PREFIX,
                                        0, ml, dm, st); }
       // attention over the cache (positions 0..pos, the new one included)
+      if (prefill_t0 >= 0 && ml == B && B >= kPrefillAttnMinRows) {
+        // a prefill pass: the rows are the consecutive positions prefill_t0 .. + B - 1 of one slot
+        ProfScope ps(m, PK_ATTN);
+        launches += launch_attention_prefill(m->qkv(), m->Kc, m->Vc, l, a.slot[0], prefill_t0, B,
+                                             m->attn_out(), dm, st);
+      } else {
       int max_len = 1;
       for (int r = 0; r < ml; ++r) {
         int len = a.pos[perm[r]] + 1;
@@ -309,6 +318,7 @@ static int32_t run_step(d3_model *m, const StepArgs &a, const int32_t *n, const 
       { ProfScope ps(m, PK_ATTN);
         launches += launch_attention(m->qkv(), m->Kc, m->Vc, m->sched(), l, ml, split_len, n_splits,
                                      m->lay.max_splits, m->part_o(), m->part_ml(), m->attn_out(), dm, st); }
+      }
       // output projection + residual
       g.W = m->wo[l]; g.R = dm.d; g.K = nq; g.act = m->attn_out(); g.act_stride = nq;
       g.tmap_w = tm ? &m->tm_o[l] : nullptr;
@@ -567,7 +577,7 @@ int32_t d3_load(const d3_config *cfg, const d3_weights *w, void *kv_dev, void *s
   const int64_t d = cfg->d_model, f = cfg->d_ffn;
   m->layer_bytes = 2 * ((int64_t)m->dm.qkv_rows * d + d * cfg->n_q_heads * cfg->head_dim + 3 * d * f + 2 * d);
   m->head_bytes = 2 * ((int64_t)cfg->vocab * d + d);
-  if (init_kernel_attributes() != 0) { delete m; return D3_ECUDA; }
+  if (init_kernel_attributes() != 0 || init_attention_prefill() != 0) { delete m; return D3_ECUDA; }
   // tensor-core projections: usable when the driver encodes every weight's tensor map
   m->tc.ok = tc_init() == 0;
   m->tc.act_split = reinterpret_cast<bf16 *>(m->scratch + m->lay.act_split);
@@ -645,7 +655,7 @@ int32_t d3_prefill(d3_model *m, int32_t slot, const int32_t *tokens, int32_t n_t
     }
     d3_schedule(L, 1.0, m->cfg.start_id, m->cfg.anchor, a.B, a.gi, n, lo, hi, perm, m_l, nullptr, nullptr);
     const bool last = t0 + a.B >= n_tokens;
-    int32_t rc = run_step(m, a, n, lo, hi, perm, m_l, last ? logits_dev : nullptr, ROWS_LAST, nullptr);
+    int32_t rc = run_step(m, a, n, lo, hi, perm, m_l, last ? logits_dev : nullptr, ROWS_LAST, nullptr, nullptr, t0);
     if (rc != D3_OK) return rc;
   }
   m->pos[slot] = n_tokens;

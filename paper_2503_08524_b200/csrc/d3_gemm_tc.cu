@@ -44,6 +44,8 @@ constexpr int kTileK = 64;                       // bf16 per row of a stage = 12
 constexpr int kABytes = kTileM * kTileK * 2;     // 16 KB
 constexpr int kMaxStagesTc = 8;
 constexpr int kSmemBudget = 100 * 1024;          // two CTAs per SM stay resident
+constexpr int kSmemBudgetWide = 200 * 1024;      // more than 64 rows: one CTA per SM, stages of 64 KB
+constexpr int kGroupRows = 64;                   // activation rows of one operand group (UMMA N = 192)
 
 static_assert(sizeof(TMap) == sizeof(CUtensorMap), "opaque tensor-map storage");
 
@@ -75,8 +77,9 @@ __device__ __forceinline__ uint32_t bar_try_wait(uint32_t bar, uint32_t parity) 
 
 struct TcArgs {
   int R, K;              // weight rows (outputs), reduction length
-  int NP;                // padded activation rows, a multiple of 8
+  int NP;                // padded activation rows of one operand group, a multiple of 8 (<= 64)
   int N;                 // UMMA N = 3 NP rounded up to a multiple of 16 (the spare columns are not read)
+  int groups;            // operand groups (1, or 2 for 65..128 rows): one MMA and N TMEM columns each
   int n_kb, kb_per_split;
   int n_stages, tmem_cols;
   int atomic;            // combine with red.add (split-K or residual)
@@ -198,7 +201,8 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
   const int n_it = kb1 - kb0;
   const int S = t.n_stages;
   const int N = t.N;
-  const uint32_t stage_bytes = (uint32_t)(kABytes + N * kTileK * 2);
+  const int G = t.groups;
+  const uint32_t stage_bytes = (uint32_t)(kABytes + G * N * kTileK * 2);
   // the swizzle pattern is a function of the address: tiles start on 1024-byte boundaries
   const uint32_t ring = (smem_addr(tc_smem_raw) + 1023u) & ~1023u;
   volatile int *abort_flag = &s_abort;
@@ -247,7 +251,9 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
       pdl_wait();                            // the activations come from the previous kernel
       for (int it = 0; it < first; ++it) {
         const uint32_t a = ring + (uint32_t)it * stage_bytes;
-        tma_load_2d(a + kABytes, &map_act, (kb0 + it) * kTileK, 0, smem_addr(&s_full[it]));
+        for (int g = 0; g < G; ++g)
+          tma_load_2d(a + kABytes + g * N * kTileK * 2, &map_act, (kb0 + it) * kTileK, g * N,
+                      smem_addr(&s_full[it]));
         issued = it + 1;
       }
       for (int it = first; it < n_it; ++it) {
@@ -260,7 +266,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
         bar_expect_tx(full, stage_bytes);
         tma_load_2d(a, &map_w0, x, row_a, full);
         tma_load_2d(a + kBoxRows * kTileK * 2, &map_w1, x, row_b, full);
-        tma_load_2d(a + kABytes, &map_act, x, 0, full);
+        for (int g = 0; g < G; ++g) tma_load_2d(a + kABytes + g * N * kTileK * 2, &map_act, x, g * N, full);
         issued = it + 1;
       }
       if (*abort_flag) {
@@ -282,10 +288,14 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
         if (!ok) break;
         fence_after_sync();
         const uint32_t a = ring + (uint32_t)s * stage_bytes;
-        const uint64_t adesc = smem_desc_sw128(a), bdesc = smem_desc_sw128(a + kABytes);
+        const uint64_t adesc = smem_desc_sw128(a);
+        for (int g = 0; g < G; ++g) {
+          const uint64_t bdesc = smem_desc_sw128(a + kABytes + g * N * kTileK * 2);
 #pragma unroll
-        for (int k = 0; k < kTileK / 16; ++k)   // 16 bf16 = 32 bytes = 2 descriptor units per MMA
-          umma_bf16(tmem, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), idesc, (it | k) ? 1u : 0u);
+          for (int k = 0; k < kTileK / 16; ++k)   // 16 bf16 = 32 bytes = 2 descriptor units per MMA
+            umma_bf16(tmem + (uint32_t)(g * N), adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), idesc,
+                      (it | k) ? 1u : 0u);
+        }
         umma_commit(smem_addr(&s_empty[s]));
       }
       umma_commit(smem_addr(&s_accum));
@@ -307,14 +317,15 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
     const bool live = *abort_flag == 0;
     int r0, r1;
     row_span(t.sched, t.layer, t.row_mode, r0, r1);
-    const int nrows = min(r1 - r0, t.NP);
+    const int nrows = min(r1 - r0, G * t.NP);
     const uint32_t tbase = tmem + ((uint32_t)(q * 32) << 16);
-    float *xch = reinterpret_cast<float *>(tc_smem_raw + (ring - smem_addr(tc_smem_raw)));   // [NP][64], SwiGLU
+    // activation row j sits in operand group j / NP at TMEM columns (j / NP) * N + j % NP (+ NP, + 2 NP)
+    float *xch = reinterpret_cast<float *>(tc_smem_raw + (ring - smem_addr(tc_smem_raw)));   // [G NP][64], SwiGLU
     if (EPI == EPI_SWIGLU) {
       if (live && trow >= kBoxRows) {
         for (int j0 = 0; j0 < nrows; j0 += 8) {
           float y[8];
-          tmem_sum3(tbase, j0, t.NP, y);
+          tmem_sum3(tbase + (uint32_t)((j0 / t.NP) * N), j0 % t.NP, t.NP, y);
 #pragma unroll
           for (int i = 0; i < 8; ++i) xch[(j0 + i) * kBoxRows + (trow - kBoxRows)] = y[i];
         }
@@ -324,7 +335,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
       if (live && trow < kBoxRows) {
         for (int j0 = 0; j0 < nrows; j0 += 8) {
           float y[8];
-          tmem_sum3(tbase, j0, t.NP, y);
+          tmem_sum3(tbase + (uint32_t)((j0 / t.NP) * N), j0 % t.NP, t.NP, y);
 #pragma unroll
           for (int i = 0; i < 8; ++i) {
             const int j = j0 + i;
@@ -339,7 +350,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
       const int r = blockIdx.x * kTileM + trow;
       for (int j0 = 0; j0 < nrows; j0 += 8) {
         float y[8];
-        tmem_sum3(tbase, j0, t.NP, y);
+        tmem_sum3(tbase + (uint32_t)((j0 / t.NP) * N), j0 % t.NP, t.NP, y);
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
           const int j = j0 + i;
@@ -371,7 +382,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
 // zeroes that output row.
 struct SplitArgs {
   const float *act;
-  int act_stride, K, NP;
+  int act_stride, K, NP, N, groups;   // NP rows per operand group, groups of N operand rows each
   const bf16 *gain;
   float eps;
   bf16 *dst;             // [3 NP][K]
@@ -392,7 +403,7 @@ __global__ void __launch_bounds__(256) k_act_split(const SplitArgs a) {
   int r0, r1;
   row_span(a.sched, a.layer, a.row_mode, r0, r1);
   const int j = blockIdx.x, row = r0 + j;
-  if (row >= r1 || j >= a.NP) return;
+  if (row >= r1 || j >= a.groups * a.NP) return;
   const float *src = a.act + (size_t)row * a.act_stride;
   float sc = 1.f;
   if (a.gain) {
@@ -413,8 +424,9 @@ __global__ void __launch_bounds__(256) k_act_split(const SplitArgs a) {
     __syncthreads();
     sc = s_scale;
   }
-  bf16 *hi = a.dst + (size_t)j * a.K, *mid = a.dst + (size_t)(a.NP + j) * a.K,
-       *lo = a.dst + (size_t)(2 * a.NP + j) * a.K;
+  const int grow = (j / a.NP) * a.N + j % a.NP;   // the row's hi term in its operand group
+  bf16 *hi = a.dst + (size_t)grow * a.K, *mid = a.dst + (size_t)(a.NP + grow) * a.K,
+       *lo = a.dst + (size_t)(2 * a.NP + grow) * a.K;
   const int k = blockIdx.y * 1024 + tid * 4;
   if (k < a.K) {
     float4 v = *reinterpret_cast<const float4 *>(src + k);
@@ -477,7 +489,8 @@ bool encode_map(TMap *out, const void *base, int rows, int K, int box_rows) {
 
 template <int EPI>
 cudaError_t tc_attr() {
-  return cudaFuncSetAttribute(k_gemm_tc<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget + 1024);
+  return cudaFuncSetAttribute(k_gemm_tc<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              kSmemBudgetWide + 1024);
 }
 
 }  // namespace
@@ -503,13 +516,17 @@ int launch_gemm_tc(TcContext &tc, const GemvArgs &g, int epi, int m_rows, cudaSt
   if (epi == EPI_SWIGLU && !g.tmap_w2) return 0;
   // three operand rows per activation row; UMMA M = 128 wants N a multiple of 16 (<= 192 here):
   // up to 8 spare rows of the operand buffer ride along (whatever they hold, their columns are unused)
-  const int NP = (m_rows + 7) / 8 * 8, N = (3 * NP + 15) / 16 * 16;
-  if ((size_t)N * g.K * sizeof(bf16) > tc.act_bytes) return 0;
-  const uint64_t key = ((uint64_t)NP << 32) | (uint32_t)g.K;
+  // More than 64 rows: two operand groups of 64 rows (N = 192 each, one MMA per group and k-step,
+  // the weight tile read from shared memory by both), so that a pass of up to 128 prompt
+  // positions streams the weights once.
+  const int groups = m_rows > kGroupRows ? 2 : 1;
+  const int NP = groups > 1 ? kGroupRows : (m_rows + 7) / 8 * 8, N = (3 * NP + 15) / 16 * 16;
+  if ((size_t)groups * N * g.K * sizeof(bf16) > tc.act_bytes) return 0;
+  const uint64_t key = ((uint64_t)groups << 48) | ((uint64_t)NP << 32) | (uint32_t)g.K;
   auto it = tc.act_maps.find(key);
   if (it == tc.act_maps.end()) {
     TMap mp;
-    if (!encode_map(&mp, tc.act_split, N, g.K, N)) return 0;
+    if (!encode_map(&mp, tc.act_split, groups * N, g.K, N)) return 0;
     it = tc.act_maps.emplace(key, mp).first;
   }
 
@@ -519,7 +536,7 @@ int launch_gemm_tc(TcContext &tc, const GemvArgs &g, int epi, int m_rows, cudaSt
   int ksplit = 1;
   if (epi == EPI_STORE || epi == EPI_RESID) {
     // all CTAs resident at once (two per SM), slices of at least 8 k-blocks
-    ksplit = 2 * tc.sm_count / tiles;
+    ksplit = (groups > 1 ? 1 : 2) * tc.sm_count / tiles;
     if (ksplit > n_kb / 8) ksplit = n_kb / 8;
     if (ksplit < 1) ksplit = 1;
     if (ksplit > 16) ksplit = 16;
@@ -528,7 +545,8 @@ int launch_gemm_tc(TcContext &tc, const GemvArgs &g, int epi, int m_rows, cudaSt
   ksplit = (n_kb + per - 1) / per;   // no empty slice
 
   SplitArgs sa;
-  sa.act = g.act; sa.act_stride = g.act_stride; sa.K = g.K; sa.NP = NP; sa.gain = g.gain; sa.eps = g.eps;
+  sa.act = g.act; sa.act_stride = g.act_stride; sa.K = g.K; sa.NP = NP; sa.N = N; sa.groups = groups;
+  sa.gain = g.gain; sa.eps = g.eps;
   sa.dst = tc.act_split;
   sa.zero_out = (epi == EPI_STORE && ksplit > 1) ? g.out : nullptr;
   sa.out_stride = g.out_stride; sa.out_col0 = g.out_col0; sa.R = g.R;
@@ -536,16 +554,16 @@ int launch_gemm_tc(TcContext &tc, const GemvArgs &g, int epi, int m_rows, cudaSt
   launch_pdl(k_act_split, dim3(m_rows, (g.K + 1023) / 1024), dim3(256), 0, st, sa);
 
   TcArgs t;
-  t.R = g.R; t.K = g.K; t.NP = NP; t.N = N; t.n_kb = n_kb; t.kb_per_split = per;
-  const int stage_bytes = kABytes + N * kTileK * 2;
-  t.n_stages = kSmemBudget / stage_bytes;
+  t.R = g.R; t.K = g.K; t.NP = NP; t.N = N; t.groups = groups; t.n_kb = n_kb; t.kb_per_split = per;
+  const int stage_bytes = kABytes + groups * N * kTileK * 2;
+  t.n_stages = (groups > 1 ? kSmemBudgetWide : kSmemBudget) / stage_bytes;
   if (t.n_stages > kMaxStagesTc) t.n_stages = kMaxStagesTc;
   // Measured: a fifth stage does not shorten any launch, but its shared memory keeps the next
   // kernel's CTAs from becoming resident early (13B shape, 8 rows: 7.24 ms per step with 5, 6.43 with 4).
   if (t.n_stages > 4) t.n_stages = 4;
   if (t.n_stages > per) t.n_stages = per < 2 ? 2 : per;
   t.tmem_cols = 32;
-  while (t.tmem_cols < N) t.tmem_cols *= 2;
+  while (t.tmem_cols < groups * N) t.tmem_cols *= 2;
   t.atomic = (epi == EPI_RESID || (epi == EPI_STORE && ksplit > 1)) ? 1 : 0;
   t.out = g.out; t.out_stride = g.out_stride; t.out_col0 = g.out_col0;
   t.sched = g.sched; t.status = const_cast<DevSched *>(g.sched); t.layer = g.layer; t.row_mode = g.row_mode;

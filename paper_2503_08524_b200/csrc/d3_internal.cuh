@@ -196,6 +196,9 @@ int launch_attention(const float *qkv, const bf16 *Kc, const bf16 *Vc, const Dev
                      int m_rows, int split_len, int n_splits, int max_splits, float *part_o,
                      float *part_ml, float *attn_out, const Dims &dm, cudaStream_t st);
 int init_attention_mma();
+int init_attention_prefill();
+int launch_attention_prefill(const float *qkv, const bf16 *Kc, const bf16 *Vc, int layer, int slot, int t0, int B,
+                             float *attn_out, const Dims &dm, cudaStream_t st);
 int launch_attention_partial_mma(const float *qkv, const bf16 *Kc, const bf16 *Vc, const DevSched *s, int layer,
                                  int m_rows, int split_len, int n_splits, int max_splits, float *part_o,
                                  float *part_ml, float *attn_out, const Dims &dm, cudaStream_t st);

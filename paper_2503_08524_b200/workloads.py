@@ -66,7 +66,7 @@ def run_workload(name, layers=0, steps=0, warmup=3, alpha=0.0, gen_offset=0, exe
     start_id = int(0.2 * shape.n_layers)
     w = I.make_weights(shape, seed, device=device)
     extra = 2 * (K * reps + W) + 16
-    model = B.D3Model(shape, w, rows, phi + extra, max(rows, 32), start_id=start_id, device=device)
+    model = B.D3Model(shape, w, rows, phi + extra, 128, start_id=start_id, device=device)
     model.zero_kv()
     lens = I.uniform_ints(seed, 3, rows, plo, phi)
     stream = torch.cuda.current_stream()

@@ -74,7 +74,7 @@ def test_host_schedule_equals_oracle(anchor):
 
 def test_schedule_rejects_bad_arguments():
     for kw in [dict(L=0), dict(L=129), dict(alpha=0.0), dict(alpha=float("nan")), dict(start_id=33),
-               dict(start_id=-1), dict(anchor=2), dict(gen_index=[-1]), dict(gen_index=[1] * 65)]:
+               dict(start_id=-1), dict(anchor=2), dict(gen_index=[-1]), dict(gen_index=[1] * 129)]:
         args = dict(L=32, alpha=0.9, start_id=6, anchor=0, gen_index=[1, 2])
         args.update(kw)
         with pytest.raises(B.D3Error) as e:
@@ -88,7 +88,7 @@ def test_workspace_and_load_validation():
     assert kv == 2 * 32 * 1 * 32 * 1024 * 128 * 2
     assert scratch > 0 and scratch % 256 == 0
     for field, bad in [("struct_size", 4), ("n_layers", 0), ("n_layers", 129), ("d_model", 4100),
-                       ("head_dim", 96), ("n_kv_heads", 5), ("max_batch", 65), ("start_id", 33),
+                       ("head_dim", 96), ("n_kv_heads", 5), ("max_batch", 129), ("start_id", 33),
                        ("anchor", 7), ("kv_fill", 3), ("kv_layout", 1), ("d_ffn", 11009)]:
         c = B.make_config(I.LLAMA_7B, 1, 1024, 1)
         setattr(c, field, bad)
