@@ -64,8 +64,7 @@ extern "C" {
                                the sequence's tokens stop running it (Sec. 3.2 leaves those
                                states undefined; nothing reads them while depth only decays).
                                Page 0 is reserved and zero-filled by d3_load: it stands in
-                               for every page never written.  Decode steps of a paged model
-                               always run as the sequence of kernels.                       */
+                               for every page never written.                                */
 
 typedef struct d3_config {
   uint32_t struct_size;     /* sizeof(d3_config), checked                              */
@@ -222,7 +221,7 @@ int32_t d3_read_kv(d3_model *m, int32_t layer, int32_t slot, int32_t pos, float 
 
 /* How decode steps execute.  AUTO: a batch of one row runs as a single persistent
  * cooperative kernel when the device and sizes allow it (fill modes NONE and
- * COPY, contiguous cache, at most 512 MiB of weights per block: beyond that the
+ * COPY, contiguous or paged cache, at most 512 MiB of weights per block: beyond that the
  * kernel sequence measured as fast or faster); everything else runs as a sequence
  * of kernels per block whose projections run on the tensor cores (tcgen05,
  * activations split exactly into three bf16 terms, fp32 accumulate) for depth

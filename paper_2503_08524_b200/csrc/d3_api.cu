@@ -292,7 +292,9 @@ static int32_t run_step(d3_model *m, const StepArgs &a, const int32_t *n, const 
       g.tmap_w = tm ? &m->tm_qkv[l] : nullptr; g.tmap_w2 = nullptr;
       g.act = m->x(); g.act_stride = dm.d; g.gain = m->attn_norm[l];
       g.out = m->qkv(); g.out_stride = dm.qkv_rows; g.out_col0 = 0;
+      g.short_chain_row0 = prefill_t0 >= 0 ? nq : 0;   // a prompt's K and V rows: see launch_gemm_tc
       { ProfScope ps(m, PK_QKV); launches += project(m, g, EPI_STORE, ml); }
+      g.short_chain_row0 = 0;
       { ProfScope ps(m, PK_ROPE);
         launches += launch_rope_append(m->qkv(), m->rope(), m->Kc, m->Vc, m->sched(), l, ROWS_PREFIX,
                                        0, ml, dm, st); }
@@ -383,7 +385,13 @@ static int32_t run_step(d3_model *m, const StepArgs &a, const int32_t *n, const 
 }
 
 // One batch-1 step as a single cooperative kernel.
-static int32_t run_fused_step(d3_model *m, const StepArgs &a, float *logits_dev, int32_t *launches_out) {
+static int32_t run_fused_step(d3_model *m, const StepArgs &a, const int32_t *lo, const int32_t *hi,
+                              float *logits_dev, int32_t *launches_out) {
+  int32_t table_launches = 0;
+  {
+    int32_t rc = pages_for_step(m, 1, a.slot, a.pos, lo, hi, &table_launches);   // paged cache: before any launch
+    if (rc != D3_OK) return rc;
+  }
   FusedParams fp;
   memset(&fp, 0, sizeof(fp));
   fp.slot = a.slot[0]; fp.tok = a.tok[0]; fp.gi = a.gi[0]; fp.pos = a.pos[0]; fp.tok_dev = a.tok_dev;
@@ -412,7 +420,7 @@ static int32_t run_fused_step(d3_model *m, const StepArgs &a, float *logits_dev,
   m->last_B = 1;
   m->last_perm[0] = 0;
   prof_collect(m);
-  if (launches_out) *launches_out = 1;
+  if (launches_out) *launches_out = 1 + table_launches;
   return (rc == 1 && cudaGetLastError() == cudaSuccess) ? D3_OK : D3_ECUDA;
 }
 
@@ -619,7 +627,6 @@ int32_t d3_load(const d3_config *cfg, const d3_weights *w, void *kv_dev, void *s
   }
   m->fused_ok = fused_plan(*cfg, &m->fused_grid, &m->fused_stages, &m->fused_act, &m->fused_smem,
                            &m->fused_func);
-  if (cfg->kv_layout != D3_KV_CONTIGUOUS) m->fused_ok = 0;   // the single-kernel step addresses a contiguous cache
   if (m->fused_ok && m->fused_grid > kFusedMaxCtas) m->fused_grid = kFusedMaxCtas;
   if (cudaMemsetAsync(m->sched(), 0, sizeof(DevSched), m->stream) != cudaSuccess ||
       cudaMemsetAsync(m->scratch + m->lay.phase, 0, (size_t)kFusedMaxCtas * kFusedPhases * 8, m->stream) !=
@@ -704,7 +711,7 @@ static int32_t decode_rows(d3_model *m, int32_t batch, const int32_t *slots, con
   const bool fused = batch == 1 && m->fused_ok &&
                      ((m->exec_mode == D3_EXEC_AUTO && small_blocks) || m->exec_mode == D3_EXEC_FUSED) &&
                      c.kv_fill != D3_FILL_RECOMPUTE && !probe;
-  int32_t rc = fused ? run_fused_step(m, a, logits_dev, &launches)
+  int32_t rc = fused ? run_fused_step(m, a, lo, hi, logits_dev, &launches)
                      : run_step(m, a, n, lo, hi, perm, m_l, logits_dev, ROWS_ALL, &launches, probe);
   if (rc != D3_OK) return rc;
   if (stats) {

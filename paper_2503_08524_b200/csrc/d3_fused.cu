@@ -320,12 +320,17 @@ struct Producer {
       for (int chunk = ch0; chunk < ch1; ++chunk) {
         if (chunk == a.nch - 1) continue;   // the chunk with the current position: plain loads
         if (!mine()) { ++s; continue; }
-        const size_t off = ((((size_t)layer * dm.max_slots + p.slot) * dm.Hkv + kvh) * dm.max_seq +
-                            (size_t)chunk * a.CH) * dm.dh;
+        // A chunk is one run of the cache, or (paged cache with pages shorter than a chunk) one
+        // run per page: lanes 2j and 2j + 1 copy K and V of run j.  Pages hold a power of two of
+        // positions and chunks start at multiples of their length, so no run straddles a page.
+        const int run_pos = (dm.page_size == 0 || dm.page_size >= a.CH) ? a.CH : dm.page_size;
+        const int n_run = a.CH / run_pos, j = lane >> 1;
+        const uint32_t run_bytes = (uint32_t)(run_pos * dm.dh * 2);
+        const size_t off = j < n_run ? kv_offset(dm, dm.block_table, layer, p.slot, kvh, chunk * a.CH + j * run_pos) : 0;
+        const bf16 *src = ((lane & 1) ? p.Vc : p.Kc) + off;
         if (l2_only) {
           if (!throttle()) return;
-          if (lane == 0) l2_prefetch(p.Kc + off, kStageBytes / 2);
-          if (lane == 1) l2_prefetch(p.Vc + off, kStageBytes / 2);
+          if (j < n_run) l2_prefetch(src, run_bytes);
           ++s;
           continue;
         }
@@ -334,9 +339,9 @@ struct Producer {
         if (pid == 0 && lane == 0) *c.progress = s;
         const uint32_t bar = smem_u32(&c.full[slot]);
         const uint32_t dst = smem_u32(c.ring + (size_t)slot * kStageBytes);
+        // (bytes may complete before the expect_tx lands: the phase cannot end before its one arrival)
         if (lane == 0) mbar_expect_tx(bar, (uint32_t)kStageBytes);
-        if (lane == 0) bulk_g2s(dst, p.Kc + off, kStageBytes / 2, bar);
-        if (lane == 1) bulk_g2s(dst + kStageBytes / 2, p.Vc + off, kStageBytes / 2, bar);
+        if (j < n_run) bulk_g2s(dst + (lane & 1) * (kStageBytes / 2) + j * run_bytes, src, run_bytes, bar);
         ++s;
       }
     }
@@ -525,7 +530,6 @@ struct Consumer {
     if (ph.kind == PH_QKV) {
       const int per_head = dm.dh / 4, half = dm.dh / 2;
       const int rot_groups = (dm.Hq + dm.Hkv) * per_head;
-      const size_t cbase = ((size_t)layer * dm.max_slots + p.slot) * dm.Hkv;
       if (g < rot_groups) {
         const int head = g / per_head, jj = (g % per_head) * 2;
         const float2 cs0 = c.rope_row[jj], cs1 = c.rope_row[jj + 1];
@@ -535,13 +539,13 @@ struct Consumer {
           float *q = p.qkv + head * dm.dh;
           q[jj] = a0; q[jj + 1] = a1; q[jj + half] = b0; q[jj + half + 1] = b1;
         } else {
-          bf16 *dst = p.Kc + ((cbase + (head - dm.Hq)) * dm.max_seq + p.pos) * dm.dh;
+          bf16 *dst = p.Kc + kv_offset(dm, dm.block_table, layer, p.slot, head - dm.Hq, p.pos);
           dst[jj] = __float2bfloat16_rn(a0); dst[jj + 1] = __float2bfloat16_rn(a1);
           dst[jj + half] = __float2bfloat16_rn(b0); dst[jj + half + 1] = __float2bfloat16_rn(b1);
         }
       } else {
         const int r = (g - rot_groups) * 4, h = r / dm.dh, e = r % dm.dh;
-        bf16 *dst = p.Vc + ((cbase + h) * dm.max_seq + p.pos) * dm.dh + e;
+        bf16 *dst = p.Vc + kv_offset(dm, dm.block_table, layer, p.slot, h, p.pos) + e;
         dst[0] = __float2bfloat16_rn(y0); dst[1] = __float2bfloat16_rn(y1);
         dst[2] = __float2bfloat16_rn(y2); dst[3] = __float2bfloat16_rn(y3);
       }
@@ -619,12 +623,12 @@ struct Consumer {
         const int t0 = chunk * a.CH;
         const int cnt = tail ? (p.pos - t0 + 1) : (mine ? a.CH : 0);
         const int i0 = tail ? worker : (lane >> 3), istep = tail ? 32 : 4;
-        const size_t goff = ((((size_t)layer * dm.max_slots + p.slot) * dm.Hkv + kvh) * dm.max_seq + t0) * DH;
         for (int i = i0; i < cnt; i += istep) {
           float kf[EPL], vf[EPL];
           if (tail) {
-            const bf16 *kp = p.Kc + goff + (size_t)i * DH + part8 * EPL;
-            const bf16 *vp = p.Vc + goff + (size_t)i * DH + part8 * EPL;
+            const size_t goff = kv_offset(dm, dm.block_table, layer, p.slot, kvh, t0 + i) + part8 * EPL;
+            const bf16 *kp = p.Kc + goff;
+            const bf16 *vp = p.Vc + goff;
 #pragma unroll
             for (int e = 0; e < EPL; e += 4) {
               const uint2 kw = __ldcg(reinterpret_cast<const uint2 *>(kp + e));
@@ -971,12 +975,12 @@ __global__ void __launch_bounds__(kFusedThreads, 1) k_step_b1(const __grid_const
     for (int l = lo + c.cta; l < hi; l += c.ncta) {
       for (int i = tid; i < nkv; i += kConsumers) {
         const int h = i / dm.dh, e = i % dm.dh;
-        const size_t dst = ((((size_t)l * dm.max_slots + p.slot) * dm.Hkv + h) * dm.max_seq + p.pos) * dm.dh + e;
+        const size_t dst = kv_offset(dm, dm.block_table, l, p.slot, h, p.pos) + e;
         if (lo == 0) {
           Ku[dst] = 0;
           Vu[dst] = 0;
         } else {
-          const size_t src = ((((size_t)(lo - 1) * dm.max_slots + p.slot) * dm.Hkv + h) * dm.max_seq + p.pos) * dm.dh + e;
+          const size_t src = kv_offset(dm, dm.block_table, lo - 1, p.slot, h, p.pos) + e;
           Ku[dst] = __ldcg(Ku + src);   // written by another CTA earlier in this kernel
           Vu[dst] = __ldcg(Vu + src);
         }

@@ -29,6 +29,8 @@
 // Every mbarrier wait is bounded in time; on expiry the CTA raises D3_ETIMEOUT in
 // the schedule's status word, stops issuing, waits (bounded) for its copies in
 // flight, frees its TMEM columns and returns.
+#include <stdlib.h>
+
 #include <cuda.h>   // CUtensorMap and its enums; the encoder is fetched at run time
 
 #include "d3_internal.cuh"
@@ -46,6 +48,7 @@ constexpr int kMaxStagesTc = 8;
 constexpr int kSmemBudget = 100 * 1024;          // two CTAs per SM stay resident
 constexpr int kSmemBudgetWide = 200 * 1024;      // more than 64 rows: one CTA per SM, stages of 64 KB
 constexpr int kGroupRows = 64;                   // activation rows of one operand group (UMMA N = 192)
+constexpr int kShortChainKb = 4;                 // k-blocks (of 4 MMAs) per slice of a short accumulation chain
 
 static_assert(sizeof(TMap) == sizeof(CUtensorMap), "opaque tensor-map storage");
 
@@ -81,6 +84,9 @@ struct TcArgs {
   int N;                 // UMMA N = 3 NP rounded up to a multiple of 16 (the spare columns are not read)
   int groups;            // operand groups (1, or 2 for 65..128 rows): one MMA and N TMEM columns each
   int n_kb, kb_per_split;
+  // tiles that end at or before row `short_row0` keep long accumulation chains: they use only the
+  // first `splits_long` slices of `kb_long` k-blocks each (the other slices of such a tile exit at once)
+  int short_row0, splits_long, kb_long;
   int n_stages, tmem_cols;
   int atomic;            // combine with red.add (split-K or residual)
   float *out;
@@ -192,8 +198,10 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
   __shared__ int s_abort;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int kb0 = blockIdx.y * t.kb_per_split;
-  const int kb1 = min(t.n_kb, kb0 + t.kb_per_split);
+  const bool long_tile = (int)(blockIdx.x + 1) * kTileM <= t.short_row0;
+  const int per_slice = long_tile ? t.kb_long : t.kb_per_split;
+  const int kb0 = (long_tile && (int)blockIdx.y >= t.splits_long) ? t.n_kb : blockIdx.y * per_slice;
+  const int kb1 = min(t.n_kb, kb0 + per_slice);
   if (kb0 >= kb1) {         // uniform over the CTA; the host launches no such slice
     pdl_wait();
     return;
@@ -543,6 +551,27 @@ int launch_gemm_tc(TcContext &tc, const GemvArgs &g, int epi, int m_rows, cudaSt
   }
   int per = (n_kb + ksplit - 1) / ksplit;
   ksplit = (n_kb + per - 1) / per;   // no empty slice
+  // Rows from g.short_chain_row0 on (the K and V rows of a prefill pass, which end up rounded to
+  // bf16 in the cache) are summed in slices of at most kShortChainKb k-blocks: the error of the
+  // tensor core's fp32 accumulation grows with the length of the chain; with chains of 32 MMAs the
+  // cached values round like those of the fp32-FMA kernels, with 16 a little better (measured
+  // through the logits of a 32-block model).  Tiles above keep `ksplit`.
+  int splits_long = ksplit, kb_long = per;
+  int short_row0 = g.R;
+  if (epi == EPI_STORE && g.short_chain_row0 > 0 && g.short_chain_row0 < g.R && n_kb > kShortChainKb) {
+    int chain = kShortChainKb;
+    if (const char *env = getenv("D3_TC_SHORT_KB")) {   // tuning knob
+      const int v = atoi(env);
+      if (v >= 2 && v <= 64) chain = v;
+    }
+    int want = (n_kb + chain - 1) / chain;
+    if (want > 32) want = 32;
+    if (want > ksplit) {
+      short_row0 = g.short_chain_row0 / kTileM * kTileM;
+      per = (n_kb + want - 1) / want;
+      ksplit = (n_kb + per - 1) / per;
+    }
+  }
 
   SplitArgs sa;
   sa.act = g.act; sa.act_stride = g.act_stride; sa.K = g.K; sa.NP = NP; sa.N = N; sa.groups = groups;
@@ -555,6 +584,7 @@ int launch_gemm_tc(TcContext &tc, const GemvArgs &g, int epi, int m_rows, cudaSt
 
   TcArgs t;
   t.R = g.R; t.K = g.K; t.NP = NP; t.N = N; t.groups = groups; t.n_kb = n_kb; t.kb_per_split = per;
+  t.short_row0 = short_row0; t.splits_long = splits_long; t.kb_long = kb_long;
   const int stage_bytes = kABytes + groups * N * kTileK * 2;
   t.n_stages = (groups > 1 ? kSmemBudgetWide : kSmemBudget) / stage_bytes;
   if (t.n_stages > kMaxStagesTc) t.n_stages = kMaxStagesTc;

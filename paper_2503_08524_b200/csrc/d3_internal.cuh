@@ -72,6 +72,7 @@ struct GemvArgs {
   float *out;
   int out_stride;
   int out_col0;         // column offset added to the output row index r
+  int short_chain_row0; // tensor-core path: rows r >= this are summed in short slices (0 = off)
   const DevSched *sched;
   int layer;
   int row_mode;

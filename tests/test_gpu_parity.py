@@ -425,15 +425,13 @@ def test_full_depth_7b_shape_against_oracle_and_between_paths(B):
     # transitions of alpha = 0.995.
     # (a) Oracle parity on a 32-token prompt.  The cache is bf16 on both sides, so a K or V
     #     element rounds differently wherever the two sides' fp values straddle a rounding
-    #     boundary; how often depends on the arithmetic that produced them.  With the prompt
-    #     projected by the fp32-FMA kernels the stated tolerances hold with a factor ~2 to spare.
-    #     With the tensor-core projections (fp32 accumulation inside tcgen05.mma, ~3x the
-    #     fp32-FMA error) about 3x as many elements round the other way: the hidden state stays 3x
-    #     inside its tolerance, the worst of the 32000 logits sits at the 2e-2 bound (measured
-    #     1.8e-2 .. 2.1e-2), so that run is held to 1.5x the logit bound.
-    # (b) At the benchmark's prompt length (512) the oracle would take minutes, so the check is a
-    #     property: the single-kernel step and the sequence of kernels (independent
-    #     implementations) agree on the same steps.
+    #     boundary; how often depends on the error of the arithmetic that produced them.  The
+    #     prompt is projected once by the fp32-FMA kernels and once by the tensor-core kernels
+    #     (whose K and V rows are summed in short chains for this reason); both runs are held to
+    #     the stated tolerances.
+    # (b) At the benchmark's prompt length (512), also a property: the single-kernel step and the
+    #     sequence of kernels (independent implementations) agree on the same steps.  (The oracle
+    #     comparison at that length is the next test.)
     shape, alpha, start = I.LLAMA_7B, 0.995, 6
     L = shape.n_layers
     orc, gpu = make_pair(shape, SEED + 11, 1, 600, 32, start_id=start, gain_jitter=0.0)
@@ -445,7 +443,7 @@ def test_full_depth_7b_shape_against_oracle_and_between_paths(B):
     o_pre = orc.prefill(0, prompt)
     ref = [orc.decode_step([0], [int(toks[k])], [i], alpha) for k, i in enumerate(gis)]
     orc.close()
-    for prefill_exec, logit_tol in ((B.EXEC_KERNELS, LOGITS_MAX_ABS), (B.EXEC_AUTO, 1.5 * LOGITS_MAX_ABS)):
+    for prefill_exec, logit_tol in ((B.EXEC_KERNELS, LOGITS_MAX_ABS), (B.EXEC_AUTO, LOGITS_MAX_ABS)):
         gpu.d3_set_exec(prefill_exec)
         gpu.d3_reset_slot(0)
         g = gpu.d3_prefill(0, prompt).cpu().numpy()
@@ -479,10 +477,37 @@ def test_full_depth_7b_shape_against_oracle_and_between_paths(B):
     gpu.close()
 
 
+def test_benchmark_configuration_against_the_oracle(B):
+    # The benchmark's own configuration against the oracle: 7B shape, all 32 blocks, batch 1,
+    # prompt of 512 tokens through the batched prefill (passes of 128 positions, as bench.py loads
+    # the model), then single-kernel decode steps at alpha = 0.995 on both sides of the depth
+    # transitions 31 -> 30 and 16 -> 15, teacher-forced.  The oracle's 512-token prefill takes a
+    # minute or two of CPU time.
+    shape, alpha, start, P = I.LLAMA_7B, 0.995, 6, 512
+    L = shape.n_layers
+    orc, gpu = make_pair(shape, SEED + 17, 1, P + 8, 128, start_id=start, gain_jitter=0.0)
+    prompt = I.prompt_tokens(shape, SEED + 17, 0, P).numpy()
+    gis = [6, 7, 138, 139]
+    toks = I.token_ids(SEED + 17, 9, len(gis), shape.vocab).numpy()
+    o_pre, o_hid = orc.prefill(0, prompt, want_hidden=True)
+    g = gpu.d3_prefill(0, prompt).cpu().numpy()
+    assert np.isfinite(g).all()
+    assert np.abs(g - o_pre).max() <= LOGITS_MAX_ABS, np.abs(g - o_pre).max()
+    assert rel_l2(gpu.d3_read_hidden(128)[(P - 1) % 128], o_hid) <= 1e-2
+    for k, i in enumerate(gis):
+        r = orc.decode_step([0], [int(toks[k])], [i], alpha)
+        gl, st = gpu.d3_decode_step([0], [int(toks[k])], [i], alpha, want_stats=True)
+        assert st["kernel_launches"] == 1 and st["n"][0] == max(O.depth(L, alpha, i), start)
+        check_step(f"i={i}", gl.cpu().numpy(), gpu.d3_read_hidden(1), r["logits"], r["hidden"])
+    gpu.d3_sync()
+    gpu.close()
+    orc.close()
+
+
 # ------------------------------------------------------------------ paged KV cache
 
 def test_paged_cache_single_row_run_and_page_accounting(B):
-    # batch 1 over a paged cache (sequence of kernels), depth decaying over page boundaries.
+    # batch 1 over a paged cache, depth decaying over page boundaries.
     # FILL_NONE never writes a dropped (token, block) pair, so a block stops taking pages once
     # the tokens stop running it; FILL_COPY writes every pair and takes pages like a dense cache.
     shape = I.TINY
@@ -520,6 +545,45 @@ def test_paged_cache_single_row_run_and_page_accounting(B):
         gpu.close()
     assert used[1] == L * 5                                          # 70 positions, dense
     assert used[0] < used[1]                                         # the depth-aware saving
+
+
+@pytest.mark.parametrize("shape,ps,fill", [(I.TINY, 16, 1), (I.TINY, 64, 0), (I.TINY, 128, 1), (I.TINY_GQA, 16, 1),
+                                           (I.TINY_GQA, 256, 0), (I.LLAMA_7B.with_layers(2), 16, 1),
+                                           (I.LLAMA_7B.with_layers(2), 32, 1)],
+                         ids=["dh64-p16", "dh64-p64-none", "dh64-p128", "dh32-gqa-p16", "dh32-gqa-p256-none",
+                              "7b-width-p16", "7b-width-p32"])
+def test_single_kernel_step_over_a_paged_cache(B, shape, ps, fill):
+    # One row over a paged cache takes the single-kernel step like a contiguous model: its
+    # producers fetch a ring stage of K and V as one run per page (pages shorter than a stage:
+    # several runs), the tail positions and the appended / filled entries go through the page table.
+    L = shape.n_layers
+    wide = shape.d_model > 1024
+    n_prompt, steps, max_seq = (150, 8, 256) if not wide else (70, 3, 128)
+    orc, gpu = make_pair(shape, SEED + 19, 2, max_seq, 8, start_id=1, kv_fill=fill, page_size=ps,
+                         n_pages=1 + L * (2 * max_seq // ps))
+    gpu.poison_kv()
+    orc.poison_kv()
+    for slot, n in ((0, n_prompt), (1, 9)):        # the second sequence interleaves its pages
+        p = I.prompt_tokens(shape, SEED + 19, slot, n).numpy()
+        o = orc.prefill(slot, p)
+        g = gpu.d3_prefill(slot, p)
+        check_step(f"prefill {slot}", g.cpu().numpy()[None], None, o[None], None)
+    toks = I.token_ids(SEED + 19, 5, 64, shape.vocab).numpy()
+    for i in range(1, steps + 1):
+        for slot in (0, 1):
+            r = orc.decode_step([slot], [int(toks[i])], [i], 0.9)
+            g, st = gpu.d3_decode_step([slot], [int(toks[i])], [i], 0.9, want_stats=True)
+            assert st["kernel_launches"] <= 2, st["kernel_launches"]     # the step, and at most one table patch
+            check_step(f"step {i} slot {slot}", g.cpu().numpy(), gpu.d3_read_hidden(1), r["logits"], r["hidden"])
+    # cache contents of the first sequence, wherever the oracle's entry is defined
+    for l in range(L):
+        for t in sorted({min(t, n_prompt + steps - 1) for t in (0, ps - 1, ps, n_prompt - 1, n_prompt, n_prompt + steps - 1)}):
+            ok, ov = orc.read_kv(l, 0, t)
+            gk, gv = gpu.d3_read_kv(l, 0, t)
+            m = np.isfinite(ok)
+            assert np.abs(gk[m] - ok[m]).max(initial=0) < 4e-2 and np.abs(gv[m] - ov[m]).max(initial=0) < 4e-2
+    gpu.d3_sync()
+    gpu.close()
 
 
 def test_paged_pool_exhaustion_is_an_error_and_changes_nothing(B):
