@@ -1,6 +1,7 @@
 // C ABI of libd3: argument validation, host bookkeeping, the host copy of the
 // depth schedule, and the per-step launch sequence.
 #include <math.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include <map>
@@ -311,7 +312,12 @@ static int32_t run_step(d3_model *m, const StepArgs &a, const int32_t *n, const 
         if (len > max_len) max_len = len;
       }
       int ctas = ml * (dm.Hq / GQ);
-      int want = (592 + ctas - 1) / ctas;
+      static const int target_ctas = [] {   // tuning knob: pieces the attention pass aims for
+        const char *env = getenv("D3_ATTN_TARGET_CTAS");
+        const int v = env ? atoi(env) : 0;
+        return v >= 148 && v <= 65536 ? v : 592;
+      }();
+      int want = (target_ctas + ctas - 1) / ctas;
       if (want < 1) want = 1;
       if (want > m->lay.max_splits) want = m->lay.max_splits;
       int split_len = ((max_len + want - 1) / want + 31) / 32 * 32;
