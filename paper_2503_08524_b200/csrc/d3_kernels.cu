@@ -635,31 +635,45 @@ int launch_table_update(int32_t *table, const TableUpdate &u, cudaStream_t st) {
 }
 
 // --------------------------------------------------------------------- argmax
+// One CTA per row: 16-byte loads, (value, index) pairs reduced by shuffles inside a warp and
+// through shared memory across warps; the lowest index wins a tie at every level.
+__device__ __forceinline__ void argmax_take(float &best, int &bi, float v, int i) {
+  if (v > best || (v == best && i < bi)) { best = v; bi = i; }
+}
+
 __global__ void __launch_bounds__(1024) k_argmax(const float *logits, int V, int32_t *out) {
   pdl_wait();
   pdl_trigger();
   const float *p = logits + (size_t)blockIdx.x * V;
   float best = -INFINITY;
   int bi = 0x7fffffff;
-  for (int i = threadIdx.x; i < V; i += blockDim.x) {
-    float v = p[i];
-    if (v > best) { best = v; bi = i; }   // strided ascending: keeps the lowest index
-  }
-  __shared__ float sv[1024];
-  __shared__ int si[1024];
-  sv[threadIdx.x] = best; si[threadIdx.x] = bi;
-  __syncthreads();
-  for (int o = blockDim.x / 2; o > 0; o >>= 1) {
-    if (threadIdx.x < o) {
-      float v2 = sv[threadIdx.x + o];
-      int i2 = si[threadIdx.x + o];
-      if (v2 > sv[threadIdx.x] || (v2 == sv[threadIdx.x] && i2 < si[threadIdx.x])) {
-        sv[threadIdx.x] = v2; si[threadIdx.x] = i2;
-      }
+  const bool vec = (V % 4 == 0) && ((reinterpret_cast<uintptr_t>(p) & 15u) == 0);
+  if (vec) {
+    for (int i = threadIdx.x * 4; i < V; i += blockDim.x * 4) {
+      const float4 v = *reinterpret_cast<const float4 *>(p + i);
+      argmax_take(best, bi, v.x, i); argmax_take(best, bi, v.y, i + 1);
+      argmax_take(best, bi, v.z, i + 2); argmax_take(best, bi, v.w, i + 3);
     }
-    __syncthreads();
+  } else {
+    for (int i = threadIdx.x; i < V; i += blockDim.x) argmax_take(best, bi, p[i], i);
   }
-  if (threadIdx.x == 0) out[blockIdx.x] = si[0] == 0x7fffffff ? 0 : si[0];
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1)
+    argmax_take(best, bi, __shfl_xor_sync(0xffffffffu, best, o), __shfl_xor_sync(0xffffffffu, bi, o));
+  __shared__ float sv[32];
+  __shared__ int si[32];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (lane == 0) { sv[warp] = best; si[warp] = bi; }
+  __syncthreads();
+  if (warp == 0) {
+    const int nw = blockDim.x >> 5;
+    best = lane < nw ? sv[lane] : -INFINITY;
+    bi = lane < nw ? si[lane] : 0x7fffffff;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1)
+      argmax_take(best, bi, __shfl_xor_sync(0xffffffffu, best, o), __shfl_xor_sync(0xffffffffu, bi, o));
+    if (lane == 0) out[blockIdx.x] = bi == 0x7fffffff ? 0 : bi;
+  }
 }
 
 // argmax and its softmax probability of one logits row; results at out[row * stride + col]

@@ -655,3 +655,12 @@ def test_argmax_lowest_index_on_ties(B):
     out = gpu.d3_argmax(lg).cpu().tolist()
     assert out == [100, 1023, 0, 0]
     gpu.close()
+    # a vocabulary that is not a multiple of four (scalar loads) and a large one, random ties
+    for vocab in (1003, 32000):
+        narrow = I.ModelShape("narrow", 1, 64, 2, 1, 32, 64, vocab)
+        orc, gpu = make_pair(narrow, SEED, 1, 8, 4)
+        g = torch.Generator().manual_seed(vocab)
+        lg = torch.randint(0, 50, (4, vocab), generator=g).float()
+        want = [int(np.flatnonzero(r == r.max())[0]) for r in lg.numpy()]
+        assert gpu.d3_argmax(lg.to("cuda:0")).cpu().tolist() == want
+        gpu.close()
