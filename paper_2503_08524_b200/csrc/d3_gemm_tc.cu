@@ -48,6 +48,7 @@ constexpr int kMaxStagesTc = 8;
 constexpr int kSmemBudget = 100 * 1024;          // two CTAs per SM stay resident
 constexpr int kSmemBudgetWide = 200 * 1024;      // more than 64 rows: one CTA per SM, stages of 64 KB
 constexpr int kGroupRows = 64;                   // activation rows of one operand group (UMMA N = 192)
+constexpr int kMaxTcRows = 2 * kGroupRows;       // activation rows of one launch
 constexpr int kShortChainKb = 4;                 // k-blocks (of 4 MMAs) per slice of a short accumulation chain
 
 static_assert(sizeof(TMap) == sizeof(CUtensorMap), "opaque tensor-map storage");
@@ -84,9 +85,10 @@ struct TcArgs {
   int N;                 // UMMA N = 3 NP rounded up to a multiple of 16 (the spare columns are not read)
   int groups;            // operand groups (1, or 2 for 65..128 rows): one MMA and N TMEM columns each
   int n_kb, kb_per_split;
-  // tiles that end at or before row `short_row0` keep long accumulation chains: they use only the
-  // first `splits_long` slices of `kb_long` k-blocks each (the other slices of such a tile exit at once)
-  int short_row0, splits_long, kb_long;
+  // CHAIN kernels: tiles that start at or after row `short_row0` sum in chains of `chain_kb` k-blocks;
+  // after each chain the epilogue warps add the accumulator to registers and the next chain starts
+  // the accumulator afresh
+  int short_row0, chain_kb;
   int n_stages, tmem_cols;
   int atomic;            // combine with red.add (split-K or residual)
   float *out;
@@ -171,6 +173,16 @@ __device__ __forceinline__ void tmem_sum3(uint32_t tbase, int j0, int NP, float 
 #pragma unroll
   for (int i = 0; i < 8; ++i) y[i] = (lo[i] + mid[i]) + hi[i];
 }
+// 16 accumulator columns of this thread's TMEM lane, without waiting for them (tmem_ld_wait does)
+__device__ __forceinline__ void tmem_ld16_issue(uint32_t taddr, uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void fence_before_sync() {
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
 }
@@ -188,20 +200,21 @@ __device__ __forceinline__ void row_span(const DevSched *s, int layer, int mode,
 }
 
 // ------------------------------------------------------------------ the GEMM
-template <int EPI>
+template <int EPI, bool CHAIN = false>
 __global__ void __launch_bounds__(kTcThreads)
 k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CUtensorMap map_w1,
           const __grid_constant__ CUtensorMap map_act, const TcArgs t) {
   extern __shared__ unsigned char tc_smem_raw[];
-  __shared__ __align__(8) uint64_t s_full[kMaxStagesTc], s_empty[kMaxStagesTc], s_accum;
+  __shared__ __align__(8) uint64_t s_full[kMaxStagesTc], s_empty[kMaxStagesTc], s_accum, s_free;
   __shared__ uint32_t s_tmem;
   __shared__ int s_abort;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const bool long_tile = (int)(blockIdx.x + 1) * kTileM <= t.short_row0;
-  const int per_slice = long_tile ? t.kb_long : t.kb_per_split;
-  const int kb0 = (long_tile && (int)blockIdx.y >= t.splits_long) ? t.n_kb : blockIdx.y * per_slice;
-  const int kb1 = min(t.n_kb, kb0 + per_slice);
+  // this tile sums in short chains (uniform over the CTA)
+  const bool chain_tile = CHAIN && (int)blockIdx.x * kTileM >= t.short_row0;
+  const int chain = chain_tile ? t.chain_kb : 0x7fffffff;
+  const int kb0 = blockIdx.y * t.kb_per_split;
+  const int kb1 = min(t.n_kb, kb0 + t.kb_per_split);
   if (kb0 >= kb1) {         // uniform over the CTA; the host launches no such slice
     pdl_wait();
     return;
@@ -221,6 +234,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
       bar_init(smem_addr(&s_empty[s]), 1);
     }
     bar_init(smem_addr(&s_accum), 1);
+    bar_init(smem_addr(&s_free), 128);   // the four epilogue warps
     s_abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -290,8 +304,18 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
     if (lane == 0) {
       const uint32_t idesc = instr_desc_bf16(kTileM, N);
       bool ok = true;
+      int chains_done = 0;   // chains committed to s_accum so far
       for (int it = 0; it < n_it && ok; ++it) {
         const int s = it % S, fill = it / S;
+        if (CHAIN && it > 0 && it % chain == 0) {
+          // the previous chain is committed; its sums must be out of the accumulator before the
+          // next chain overwrites it
+          umma_commit(smem_addr(&s_accum));
+          ok = bar_wait(smem_addr(&s_free), (uint32_t)(chains_done & 1), abort_flag, t.wait_ns, true);
+          ++chains_done;
+          if (!ok) break;
+          fence_after_sync();
+        }
         ok = bar_wait(smem_addr(&s_full[s]), (uint32_t)(fill & 1), abort_flag, t.wait_ns, true);
         if (!ok) break;
         fence_after_sync();
@@ -302,7 +326,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
 #pragma unroll
           for (int k = 0; k < kTileK / 16; ++k)   // 16 bf16 = 32 bytes = 2 descriptor units per MMA
             umma_bf16(tmem + (uint32_t)(g * N), adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), idesc,
-                      (it | k) ? 1u : 0u);
+                      ((CHAIN ? it % chain : it) | k) ? 1u : 0u);
         }
         umma_commit(smem_addr(&s_empty[s]));
       }
@@ -311,7 +335,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
         // aborted: the MMAs already issued still read shared memory and write TMEM; they end by
         // themselves, so wait for them (bounded) before the CTA gives both back
         const unsigned long long bound = t.wait_ns > kDrainFloorNs ? t.wait_ns : kDrainFloorNs;
-        bar_wait(smem_addr(&s_accum), 0u, abort_flag, bound, false);
+        bar_wait(smem_addr(&s_accum), (uint32_t)(chains_done & 1), abort_flag, bound, false);
       }
     }
     __syncwarp();
@@ -319,14 +343,65 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
     // ---------------------------------------------------------------- epilogue
     const int q = warp & 3;                   // the TMEM lane quarter this warp may read
     const int trow = q * 32 + lane;           // row of the tile = TMEM lane
-    bar_wait(smem_addr(&s_accum), 0u, abort_flag, t.wait_ns, true);
-    fence_after_sync();
-    epilogue_sync();                          // every epilogue warp sees the same abort state below
-    const bool live = *abort_flag == 0;
     int r0, r1;
     row_span(t.sched, t.layer, t.row_mode, r0, r1);
     const int nrows = min(r1 - r0, G * t.NP);
     const uint32_t tbase = tmem + ((uint32_t)(q * 32) << 16);
+    if (CHAIN && chain_tile) {
+      // ---- short chains: the row's sums live in registers, one partial sum per chain is added
+      float acc[kMaxTcRows / 16][16];
+#pragma unroll
+      for (int b = 0; b < kMaxTcRows / 16; ++b)
+#pragma unroll
+        for (int i = 0; i < 16; ++i) acc[b][i] = 0.f;
+      const int n_chains = (n_it + chain - 1) / chain;
+      bool ok = true;
+      for (int c = 0; c < n_chains && ok; ++c) {
+        ok = bar_wait(smem_addr(&s_accum), (uint32_t)(c & 1), abort_flag, t.wait_ns, true);
+        if (!ok) break;
+        fence_after_sync();
+        // 16 activation rows per trip: the three terms' columns are requested together and awaited
+        // once (a trip may read past the group's rows into columns of rows that are never written out)
+#pragma unroll
+        for (int b = 0; b < kMaxTcRows / 16; ++b) {
+          if (b * 16 < nrows) {
+            const uint32_t col = tbase + (uint32_t)(((b * 16) / t.NP) * N + (b * 16) % t.NP);
+            uint32_t hi[16], mid[16], lo[16];
+            tmem_ld16_issue(col, hi);
+            tmem_ld16_issue(col + (uint32_t)t.NP, mid);
+            tmem_ld16_issue(col + (uint32_t)(2 * t.NP), lo);
+            tmem_ld_wait();
+#pragma unroll
+            for (int i = 0; i < 16; ++i)
+              acc[b][i] += (__uint_as_float(lo[i]) + __uint_as_float(mid[i])) + __uint_as_float(hi[i]);
+          }
+        }
+        if (c + 1 < n_chains) {   // the accumulator may be overwritten
+          fence_before_sync();
+          asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(&s_free)) : "memory");
+        }
+      }
+      epilogue_sync();
+      if (*abort_flag == 0) {
+        const int r = blockIdx.x * kTileM + trow;
+#pragma unroll
+        for (int b = 0; b < kMaxTcRows / 16; ++b) {
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            const int j = b * 16 + i;
+            if (j < nrows && r < t.R) {
+              float *o = t.out + (size_t)(r0 + j) * t.out_stride + t.out_col0 + r;
+              if (t.atomic) asm volatile("red.global.add.f32 [%0], %1;" ::"l"(o), "f"(acc[b][i]) : "memory");
+              else *o = acc[b][i];
+            }
+          }
+        }
+      }
+    } else {
+    bar_wait(smem_addr(&s_accum), 0u, abort_flag, t.wait_ns, true);
+    fence_after_sync();
+    epilogue_sync();                          // every epilogue warp sees the same abort state below
+    const bool live = *abort_flag == 0;
     // activation row j sits in operand group j / NP at TMEM columns (j / NP) * N + j % NP (+ NP, + 2 NP)
     float *xch = reinterpret_cast<float *>(tc_smem_raw + (ring - smem_addr(tc_smem_raw)));   // [G NP][64], SwiGLU
     if (EPI == EPI_SWIGLU) {
@@ -371,6 +446,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
           }
         }
       }
+    }
     }
   }
 
@@ -511,6 +587,9 @@ bool tc_weight_map(TMap *out, const bf16 *W, int R, int K) {
 int tc_init() {
   if (!encoder()) return -1;
   cudaError_t e = tc_attr<EPI_STORE>();
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(k_gemm_tc<EPI_STORE, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             kSmemBudgetWide + 1024);
   if (e == cudaSuccess) e = tc_attr<EPI_RESID>();
   if (e == cudaSuccess) e = tc_attr<EPI_SWIGLU>();
   if (e == cudaSuccess) e = tc_attr<EPI_LOGITS>();
@@ -552,25 +631,20 @@ int launch_gemm_tc(TcContext &tc, const GemvArgs &g, int epi, int m_rows, cudaSt
   int per = (n_kb + ksplit - 1) / ksplit;
   ksplit = (n_kb + per - 1) / per;   // no empty slice
   // Rows from g.short_chain_row0 on (the K and V rows of a prefill pass, which end up rounded to
-  // bf16 in the cache) are summed in slices of at most kShortChainKb k-blocks: the error of the
-  // tensor core's fp32 accumulation grows with the length of the chain; with chains of 32 MMAs the
-  // cached values round like those of the fp32-FMA kernels, with 16 a little better (measured
-  // through the logits of a 32-block model).  Tiles above keep `ksplit`.
-  int splits_long = ksplit, kb_long = per;
-  int short_row0 = g.R;
-  if (epi == EPI_STORE && g.short_chain_row0 > 0 && g.short_chain_row0 < g.R && n_kb > kShortChainKb) {
-    int chain = kShortChainKb;
+  // bf16 in the cache) are summed in chains of kShortChainKb k-blocks: the error of the tensor core's
+  // fp32 accumulation grows with the length of the chain; with chains of 32 MMAs the cached values
+  // round like those of the fp32-FMA kernels, with 16 a little better (measured through the logits
+  // of a 32-block model).  The chains are summed inside the CTA (k_gemm_tc<EPI_STORE, true>): after
+  // each one the epilogue warps add the accumulator to registers.  Tiles above that row keep one chain.
+  int short_row0 = g.R, chain_kb = 0;
+  if (epi == EPI_STORE && g.short_chain_row0 > 0 && g.short_chain_row0 < g.R && per > kShortChainKb) {
+    chain_kb = kShortChainKb;
     if (const char *env = getenv("D3_TC_SHORT_KB")) {   // tuning knob
       const int v = atoi(env);
-      if (v >= 2 && v <= 64) chain = v;
+      if (v >= 2 && v <= 64) chain_kb = v;
     }
-    int want = (n_kb + chain - 1) / chain;
-    if (want > 32) want = 32;
-    if (want > ksplit) {
-      short_row0 = g.short_chain_row0 / kTileM * kTileM;
-      per = (n_kb + want - 1) / want;
-      ksplit = (n_kb + per - 1) / per;
-    }
+    short_row0 = (g.short_chain_row0 + kTileM - 1) / kTileM * kTileM;
+    if (short_row0 >= g.R) chain_kb = 0;
   }
 
   SplitArgs sa;
@@ -584,7 +658,7 @@ int launch_gemm_tc(TcContext &tc, const GemvArgs &g, int epi, int m_rows, cudaSt
 
   TcArgs t;
   t.R = g.R; t.K = g.K; t.NP = NP; t.N = N; t.groups = groups; t.n_kb = n_kb; t.kb_per_split = per;
-  t.short_row0 = short_row0; t.splits_long = splits_long; t.kb_long = kb_long;
+  t.short_row0 = short_row0; t.chain_kb = chain_kb;
   const int stage_bytes = kABytes + groups * N * kTileK * 2;
   t.n_stages = (groups > 1 ? kSmemBudgetWide : kSmemBudget) / stage_bytes;
   if (t.n_stages > kMaxStagesTc) t.n_stages = kMaxStagesTc;
@@ -604,7 +678,10 @@ int launch_gemm_tc(TcContext &tc, const GemvArgs &g, int epi, int m_rows, cudaSt
   const CUtensorMap *ma = reinterpret_cast<const CUtensorMap *>(&it->second);
   dim3 grid((unsigned)tiles, (unsigned)ksplit);
   switch (epi) {
-    case EPI_STORE: launch_pdl(k_gemm_tc<EPI_STORE>, grid, dim3(kTcThreads), smem, st, *w0, *w1, *ma, t); break;
+    case EPI_STORE:
+      if (chain_kb > 0) launch_pdl(k_gemm_tc<EPI_STORE, true>, grid, dim3(kTcThreads), smem, st, *w0, *w1, *ma, t);
+      else launch_pdl(k_gemm_tc<EPI_STORE>, grid, dim3(kTcThreads), smem, st, *w0, *w1, *ma, t);
+      break;
     case EPI_RESID: launch_pdl(k_gemm_tc<EPI_RESID>, grid, dim3(kTcThreads), smem, st, *w0, *w1, *ma, t); break;
     case EPI_SWIGLU: launch_pdl(k_gemm_tc<EPI_SWIGLU>, grid, dim3(kTcThreads), smem, st, *w0, *w1, *ma, t); break;
     default: launch_pdl(k_gemm_tc<EPI_LOGITS>, grid, dim3(kTcThreads), smem, st, *w0, *w1, *ma, t); break;
