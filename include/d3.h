@@ -221,8 +221,7 @@ int32_t d3_read_kv(d3_model *m, int32_t layer, int32_t slot, int32_t pos, float 
 
 /* How decode steps execute.  AUTO: a batch of one row runs as a single persistent
  * cooperative kernel when the device and sizes allow it (fill modes NONE and
- * COPY, contiguous or paged cache, at most 512 MiB of weights per block: beyond that the
- * kernel sequence measured as fast or faster); everything else runs as a sequence
+ * COPY, contiguous or paged cache); everything else runs as a sequence
  * of kernels per block whose projections run on the tensor cores (tcgen05,
  * activations split exactly into three bf16 terms, fp32 accumulate) for depth
  * groups of D3_TENSOR_MIN_ROWS rows or more (FP32-FMA GEMVs where the driver
@@ -233,8 +232,7 @@ int32_t d3_read_kv(d3_model *m, int32_t layer, int32_t slot, int32_t pos, float 
 #define D3_EXEC_AUTO 0
 #define D3_EXEC_KERNELS 1
 #define D3_EXEC_TENSOR 2
-#define D3_EXEC_FUSED 3    /* like AUTO, but a single row takes the single-kernel step whatever
-                              the block size (D3_EINVAL when that kernel cannot serve the model) */
+#define D3_EXEC_FUSED 3    /* like AUTO; D3_EINVAL when the single-kernel step cannot serve the model */
 #define D3_TENSOR_MIN_ROWS 1
 int32_t d3_set_exec(d3_model *m, int32_t mode);
 

@@ -709,13 +709,10 @@ static int32_t decode_rows(d3_model *m, int32_t batch, const int32_t *slots, con
   int32_t touched = 0;
   schedule_of_depths(L, c.start_id, c.anchor, batch, depth_in, n, lo, hi, perm, m_l, &rows_layers, &touched);
   int32_t launches = 0;
-  // Measured: the single kernel wins while a block's weights are small (7B shape: 2.78 ms
-  // against 3.50 ms for the kernel sequence); from the 13B shape on (634 MB per block) the
-  // tensor-core kernel sequence is as fast or faster (5.71 / 25.4 ms against 5.89 / 25.8 ms),
-  // its fixed cost per launch being small next to the streaming time.
-  const bool small_blocks = m->layer_bytes <= (512ll << 20) || !m->tm_ok;
+  // Measured (one row, full depth, same box): the single kernel wins at every shape: 7B 2.55 ms
+  // against 3.50 ms for the kernel sequence, 13B 5.47 against 5.90, 70B 25.4 against 25.7.
   const bool fused = batch == 1 && m->fused_ok &&
-                     ((m->exec_mode == D3_EXEC_AUTO && small_blocks) || m->exec_mode == D3_EXEC_FUSED) &&
+                     (m->exec_mode == D3_EXEC_AUTO || m->exec_mode == D3_EXEC_FUSED) &&
                      c.kv_fill != D3_FILL_RECOMPUTE && !probe;
   int32_t rc = fused ? run_fused_step(m, a, lo, hi, logits_dev, &launches)
                      : run_step(m, a, n, lo, hi, perm, m_l, logits_dev, ROWS_ALL, &launches, probe);

@@ -264,9 +264,8 @@ def test_production_widths(B, base, layers, Bn):
         g = gpu.d3_prefill(b, p)
         check_step(f"prefill {b}", g.cpu().numpy()[None], None, o[None], None)
     for step in range(4):
-        # single rows: the single-kernel step on even steps, whatever AUTO picks on odd ones
-        # (blocks above 512 MiB go to the tensor-core kernel sequence there)
-        gpu.d3_set_exec(B.EXEC_FUSED if (Bn == 1 and not pk and step % 2 == 0) else B.EXEC_AUTO)
+        # single rows: the single-kernel step on even steps, the tensor-core kernel sequence on odd ones
+        gpu.d3_set_exec((B.EXEC_AUTO if step % 2 == 0 else B.EXEC_TENSOR) if (Bn == 1 and not pk) else B.EXEC_AUTO)
         toks = I.token_ids(SEED + 5, 40 + step, Bn, shape.vocab).numpy()
         gi = [1 + step + 2 * b for b in range(Bn)]
         alpha = 0.8
