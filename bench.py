@@ -451,7 +451,14 @@ def main():
                     box["s"] = ClockSampler(local)
                 else:
                     box["clocks"] = box.pop("s").stop()
-            r = WL.run_workload(name, steps=24 if name != "c5" else 12, reps=3, device=dev, on_timed=on_timed)
+            try:
+                r = WL.run_workload(name, steps=24 if name != "c5" else 12, reps=3, device=dev, on_timed=on_timed)
+            except Exception as exc:     # the main line must still be printed
+                if "s" in box:
+                    box.pop("s").stop()
+                workloads[name] = {"workload": name, "error": f"{type(exc).__name__}: {exc}"[:300]}
+                torch.cuda.empty_cache()
+                continue
             r["clocks"] = box.get("clocks")
             r.pop("kernel_classes", None)
             workloads[name] = r
@@ -459,9 +466,13 @@ def main():
 
     cpu_baseline = None
     if world == 1 and not args.no_cpu_baseline:
-        w = I.make_weights(shape, I.BASE_SEED, device=dev)
-        cpu_baseline = oracle_baseline(w, shape, args.alpha, start_id, oracle_steps(K))
-        del w
+        try:
+            w = I.make_weights(shape, I.BASE_SEED, device=dev)
+            cpu_baseline = oracle_baseline(w, shape, args.alpha, start_id, oracle_steps(K))
+            del w
+        except Exception as exc:         # the main line must still be printed
+            cpu_baseline = {"value": None, "unit": "tokens/s", "cores": None, "kind": "oracle",
+                            "sample": f"failed: {type(exc).__name__}: {exc}"[:300]}
 
     line = {
         "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": K,
