@@ -49,7 +49,7 @@ ORACLE_PROMPT = 32            # bounded sample for the CPU oracle
 # ncu capture summarised in profiles/fused_step_k_step_b1_7bshape_L4.md (4-block case of the same
 # kernel: 1.8941 GB moved for 1.881 GB algorithmic; traffic grows with the blocks executed, so the
 # full launch is scaled by its own algorithmic bytes).  Set to None when the kernel changes.
-FUSED_TRAFFIC_RATIO = 1.0070
+FUSED_TRAFFIC_RATIO = None
 
 
 def gen_indices(k: int):
@@ -400,9 +400,17 @@ def main():
                 "peak_kind": f"of {peak_kind} (STREAM-style copy)", "traffic": None,
                 "share_of_kernel_time": top_ms / prof_total, "launches": top_n}
     if top_name in class_bytes:
-        ach = class_bytes[top_name] * BATCH / 1e9 / (top_ms / top_n / 1e3)
+        launch_ms = top_ms / top_n
+        timed = "per-launch CUDA events of the profiled pass (a synchronize after every step)"
+        if top_name == "fused_step" and tot["launches"] == K:
+            # one launch per step: the timed region itself (median repetition, events around its K
+            # launches back to back, the 1 KiB counter memsets included) is the launch duration
+            launch_ms = ms / K
+            timed = "CUDA events around the K launches of the timed region (median repetition)"
+        ach = class_bytes[top_name] * BATCH / 1e9 / (launch_ms / 1e3)
         roofline.update(achieved=ach, frac=ach / peak, frac_of_nominal_8TBs=ach / NOMINAL_HBM_GBS,
-                        bytes_per_launch=class_bytes[top_name], avg_launch_us=1e3 * top_ms / top_n)
+                        bytes_per_launch=class_bytes[top_name], avg_launch_us=1e3 * launch_ms,
+                        avg_launch_us_profiled_pass=1e3 * top_ms / top_n, timed=timed)
         if top_name == "fused_step" and FUSED_TRAFFIC_RATIO is not None:
             roofline["traffic"] = FUSED_TRAFFIC_RATIO * class_bytes[top_name]
     else:

@@ -407,7 +407,18 @@ __device__ void load_act_plain(const Ctx &c, const float *src, int K) {
 
 // act := RMSNorm(src) * gain.  Up to 4096 elements: one pass over L2, the values wait
 // in registers for the scale.  Wider: sum of squares first, then a second pass.
-__device__ void load_act_norm(const Ctx &c, const float *src, int K, const GainRegs &gr, const bf16 *gain) {
+// `emb` (nullable): take the vector from this bf16 row instead of `src` (the embedding row of the
+// step's token: a weight, every CTA reads it itself, nothing to wait for).
+__device__ __forceinline__ float4 ld_src4(const float *src, const bf16 *emb, int k) {
+  if (emb) {
+    const uint2 w = *reinterpret_cast<const uint2 *>(emb + k);
+    return make_float4(bfl(w.x), bfh(w.x), bfl(w.y), bfh(w.y));
+  }
+  return ldcg4(src + k);
+}
+
+__device__ void load_act_norm(const Ctx &c, const float *src, int K, const GainRegs &gr, const bf16 *gain,
+                              const bf16 *emb = nullptr) {
   const int tid = threadIdx.x;
   if (K <= GainRegs::kMaxIt * kConsumers * 4) {
     float4 v[GainRegs::kMaxIt];
@@ -416,7 +427,7 @@ __device__ void load_act_norm(const Ctx &c, const float *src, int K, const GainR
     for (int it = 0; it < GainRegs::kMaxIt; ++it) {
       const int k = it * (kConsumers * 4) + tid * 4;
       if (k < K) {
-        v[it] = ldcg4(src + k);
+        v[it] = ld_src4(src, emb, k);
         ss += v[it].x * v[it].x + v[it].y * v[it].y + v[it].z * v[it].z + v[it].w * v[it].w;
       }
     }
@@ -435,12 +446,12 @@ __device__ void load_act_norm(const Ctx &c, const float *src, int K, const GainR
   } else {
     float ss = 0.f;
     for (int k = tid * 4; k < K; k += kConsumers * 4) {
-      const float4 t = ldcg4(src + k);
+      const float4 t = ld_src4(src, emb, k);
       ss += t.x * t.x + t.y * t.y + t.z * t.z + t.w * t.w;
     }
     const float scale = rsqrtf(block_sum(ss) / (float)K + c.p->eps);
     for (int k = tid * 4; k < K; k += kConsumers * 4) {
-      float4 t = ldcg4(src + k);
+      float4 t = ld_src4(src, emb, k);
       const uint2 gw = *reinterpret_cast<const uint2 *>(gain + k);
       t.x *= scale * bfl(gw.x); t.y *= scale * bfh(gw.x);
       t.z *= scale * bfl(gw.y); t.w *= scale * bfh(gw.y);
@@ -928,12 +939,15 @@ __global__ void __launch_bounds__(kFusedThreads, 1) k_step_b1(const __grid_const
   GainRegs gr;
   const bf16 *gain = l < L ? p.layers[l].attn_norm : p.final_norm;
   prefetch_gain(gr, gain, dm.d);
-  grid_barrier(c, ++bidx);
+  consumer_sync();   // s_x_own, s_rope
   tick(0);
+  // until a block has run, the residual stream is the embedding row itself: no exchange needed
+  const bf16 *x_is_emb = emb;
   while (l < L) {
     int next = l + 1;   // dropped blocks: the hidden state passes through
     while (next < L && lo <= next && next < hi) ++next;
-    load_act_norm(c, p.x, dm.d, gr, gain);
+    load_act_norm(c, p.x, dm.d, gr, gain, x_is_emb);
+    x_is_emb = nullptr;
     tick(1);
     cs.gemv_phase(make_phase(p, PH_QKV, l, c.cta, c.ncta), l);
     tick(2);
@@ -967,7 +981,12 @@ __global__ void __launch_bounds__(kFusedThreads, 1) k_step_b1(const __grid_const
     tick(3);
     l = next;
   }
-  // KV fill by copy for the dropped blocks: CTA j takes block lo + j, lo + j + ncta, ...
+  if (p.logits) {
+    load_act_norm(c, p.x, dm.d, gr, gain, x_is_emb);
+    cs.gemv_phase(make_phase(p, PH_HEAD, 0, c.cta, c.ncta), 0);
+  }
+  // KV fill by copy for the dropped blocks: CTA j takes block lo + j, lo + j + ncta, ...  (after the
+  // LM head: nothing in this step reads the filled entries, and the head need not wait for them)
   if (p.kv_fill == D3_FILL_COPY) {
     const int nkv = dm.Hkv * dm.dh;
     unsigned short *Ku = reinterpret_cast<unsigned short *>(p.Kc);
@@ -986,10 +1005,6 @@ __global__ void __launch_bounds__(kFusedThreads, 1) k_step_b1(const __grid_const
         }
       }
     }
-  }
-  if (p.logits) {
-    load_act_norm(c, p.x, dm.d, gr, gain);
-    cs.gemv_phase(make_phase(p, PH_HEAD, 0, c.cta, c.ncta), 0);
   }
   tick(8);
   if (timing) {
