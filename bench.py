@@ -47,9 +47,9 @@ FALLBACK_HBM_GBS = 6650.0
 ORACLE_PROMPT = 32            # bounded sample for the CPU oracle
 # dram__bytes_read + dram__bytes_write of one k_step_b1 launch over its algorithmic bytes, from the
 # ncu capture summarised in profiles/fused_step_k_step_b1_7bshape_L4.md (4-block case of the same
-# kernel: 1.8941 GB moved for 1.881 GB algorithmic; traffic grows with the blocks executed, so the
+# kernel: 1.8960 GB moved for 1.881 GB algorithmic; traffic grows with the blocks executed, so the
 # full launch is scaled by its own algorithmic bytes).  Set to None when the kernel changes.
-FUSED_TRAFFIC_RATIO = None
+FUSED_TRAFFIC_RATIO = 1.0080
 
 
 def gen_indices(k: int):
