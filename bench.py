@@ -359,7 +359,7 @@ def main():
         barrier()
         e0.record(stream)
         for j in range(K):
-            model.d3_decode_step([0], [cur], [gi[j]], args.alpha, logits=logits)   # host arrays -> device
+            model.d3_decode_one(0, cur, gi[j], args.alpha, logits)                  # host arrays -> device
             model.d3_argmax(logits, tok_dev)
             if copy_logits:
                 logits_host.copy_(logits, non_blocking=True)                        # device -> host

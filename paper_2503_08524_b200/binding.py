@@ -285,6 +285,20 @@ class D3Model:
                             "algorithmic_bytes": int(st.algorithmic_bytes)}
         return logits
 
+    def d3_decode_one(self, slot: int, token: int, gen_index: int, alpha: float,
+                      logits: torch.Tensor) -> torch.Tensor:
+        """d3_decode_step for one row with the least marshalling (a greedy loop calls this once
+        per token): the three one-element arrays are kept in the object, `logits` [vocab] or
+        [1][vocab] is the caller's."""
+        a = getattr(self, "_one", None)
+        if a is None:
+            a = self._one = ((C.c_int32 * 1)(), (C.c_int32 * 1)(), (C.c_int32 * 1)())
+        a[0][0], a[1][0], a[2][0] = slot, token, gen_index
+        rc = LIB.d3_decode_step(self.h, 1, a[0], a[1], a[2], float(alpha), logits.data_ptr(), None, None)
+        if rc != OK:
+            raise D3Error(rc, "d3_decode_step")
+        return logits
+
     def d3_saturation_probe(self, slots, tokens):
         """One full-depth step; returns (logits [B][V], tokens [B][L] int32, conf [B][L] fp32),
         all on the device: what the LM head predicts from every block's output."""

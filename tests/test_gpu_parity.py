@@ -480,13 +480,13 @@ def test_benchmark_configuration_against_the_oracle(B):
     # The benchmark's own configuration against the oracle: 7B shape, all 32 blocks, batch 1,
     # prompt of 512 tokens through the batched prefill (passes of 128 positions, as bench.py loads
     # the model), then single-kernel decode steps at alpha = 0.995 on both sides of the depth
-    # transitions 31 -> 30 and 16 -> 15, teacher-forced.  The oracle's 512-token prefill takes a
+    # transition 31 -> 30 and at depth 15, teacher-forced.  The oracle's 512-token prefill takes a
     # minute or two of CPU time.
     shape, alpha, start, P = I.LLAMA_7B, 0.995, 6, 512
     L = shape.n_layers
     orc, gpu = make_pair(shape, SEED + 17, 1, P + 8, 128, start_id=start, gain_jitter=0.0)
     prompt = I.prompt_tokens(shape, SEED + 17, 0, P).numpy()
-    gis = [6, 7, 138, 139]
+    gis = [6, 7, 139]
     toks = I.token_ids(SEED + 17, 9, len(gis), shape.vocab).numpy()
     o_pre, o_hid = orc.prefill(0, prompt, want_hidden=True)
     g = gpu.d3_prefill(0, prompt).cpu().numpy()
@@ -602,6 +602,25 @@ def test_paged_pool_exhaustion_is_an_error_and_changes_nothing(B):
     r = orc.decode_step([0], [5], [1], 1.0)
     g = gpu.d3_decode_step([0], [5], [1], 1.0)
     check_step("after reset", g.cpu().numpy(), gpu.d3_read_hidden(1), r["logits"], r["hidden"])
+    gpu.d3_sync()
+    gpu.close()
+
+
+def test_single_row_call_with_the_least_marshalling(B):
+    # the greedy loop's entry of the binding: same C call, one row, against the oracle
+    shape = I.TINY
+    orc, gpu = make_pair(shape, SEED + 23, 2, 40, 2, start_id=1)
+    p = I.prompt_tokens(shape, SEED + 23, 0, 13).numpy()
+    tok = O.argmax(orc.prefill(1, p))
+    gpu.d3_prefill(1, p)
+    lg = torch.empty((1, shape.vocab), dtype=torch.float32, device="cuda:0")
+    for i in range(1, 6):
+        r = orc.decode_step([1], [tok], [i], 0.9)
+        gpu.d3_decode_one(1, tok, i, 0.9, lg)
+        check_step(f"step {i}", lg.cpu().numpy(), gpu.d3_read_hidden(1), r["logits"], r["hidden"])
+        tok = O.argmax(r["logits"][0])
+    with pytest.raises(B.D3Error):
+        gpu.d3_decode_one(0, tok, 1, 0.9, lg)      # slot 0 was never prefilled
     gpu.d3_sync()
     gpu.close()
 
