@@ -278,6 +278,34 @@ def test_production_widths(B, base, layers, Bn):
     gpu.close()
 
 
+def test_thirty_two_rows_at_7b_width_with_long_and_short_contexts(B):
+    """The batched workload's own step shape: 7B-width blocks, 32 rows in one step, contexts from a
+    few tokens up to 1024 (the attention pass then cuts the long rows into pieces and merges them),
+    retained depths mixed inside the step.  Two blocks keep the oracle's prefill of the long rows
+    to about half a minute."""
+    shape = I.LLAMA_7B.with_layers(2)
+    Bn = 32
+    orc, gpu = make_pair(shape, SEED + 21, Bn, 1040, Bn, start_id=1, kv_fill=1)
+    long_rows = {0: 1024, 5: 640, 11: 300, 18: 128, 31: 513}
+    short = I.uniform_ints(SEED + 21, 2, Bn, 3, 12)
+    for b in range(Bn):
+        n = long_rows.get(b, int(short[b]))
+        p = I.prompt_tokens(shape, SEED + 21, b, n).numpy()
+        o = orc.prefill(b, p)
+        g = gpu.d3_prefill(b, p)
+        if b in long_rows:
+            check_step(f"prefill {b}", g.cpu().numpy()[None], None, o[None], None)
+    for step in range(2):
+        toks = I.token_ids(SEED + 21, 50 + step, Bn, shape.vocab).numpy()
+        depths = [2 if (b + step) % 3 else 1 for b in range(Bn)]   # long rows on both sides of the cut
+        r = orc.decode_step_depths(list(range(Bn)), toks, depths)
+        g, st = gpu.d3_decode_step_depths(list(range(Bn)), toks, depths, want_stats=True)
+        check_step(f"step {step}", g.cpu().numpy(), gpu.d3_read_hidden(Bn), r["logits"], r["hidden"])
+        assert st["rows_layers"] == sum(depths)
+    gpu.d3_sync()
+    gpu.close()
+
+
 # ------------------------------------------------ the largest step the ABI allows
 
 def test_sixty_four_rows_per_step(B):
