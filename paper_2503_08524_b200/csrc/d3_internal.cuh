@@ -151,12 +151,13 @@ struct Layout {
 
 // Programmatic dependent launch: every kernel of the step sequence is launched
 // with the stream-serialization attribute, so that it may become resident while
-// its predecessor still runs.  EVERY thread calls pdl_wait() before it touches
+// its predecessor still runs.  Every thread calls pdl_wait() before it touches
 // anything another kernel of the stream writes or reads (it returns once all
 // earlier kernels have completed and their writes are visible); what precedes
-// the call may only touch kernel parameters, constant weights and the CTA's own
-// shared / tensor memory.  Because no CTA exits without the wait, completion of
-// a kernel implies completion of all its predecessors.
+// the call, and a thread that never makes it, may only touch kernel parameters,
+// constant weights and the CTA's own shared / tensor memory.  Because no CTA
+// exits before one of its threads has returned from the wait, completion of a
+// kernel implies completion of all its predecessors.
 #ifdef __CUDACC__
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
