@@ -248,6 +248,7 @@ static int project(d3_model *m, const GemvArgs &g, int epi, int rows) {
     int n = launch_gemm_tc(m->tc, g, epi, rows, m->stream);
     if (n) return n;
   }
+  if (g.clear) cudaMemsetAsync(g.clear, 0, g.clear_floats * sizeof(float), m->stream);   // the FMA kernels clear nothing
   return launch_gemv(g, epi, rows, m->stream);
 }
 
@@ -282,6 +283,12 @@ static int32_t run_step(d3_model *m, const StepArgs &a, const int32_t *n, const 
   memset(&g, 0, sizeof(g));
   g.sched = m->sched();
   g.eps = c.rms_eps;
+  g.clear = nullptr; g.clear_floats = 0; g.out_is_zero = 0;
+  // The QKV projection sums its k-slices into a zeroed buffer.  After a block's attention nothing
+  // reads that buffer until the next block's projection, so the down projection in between clears
+  // it on the side (decode steps without recomputed fills, which use the buffer in between).
+  const bool clear_ahead = prefill_t0 < 0 && !probe && c.kv_fill != D3_FILL_RECOMPUTE;
+  bool qkv_cleared = false;
   const bool tm = m->tm_ok;
   for (int l = 0; l < L; ++l) {
     const int ml = m_l[l];
@@ -294,8 +301,9 @@ static int32_t run_step(d3_model *m, const StepArgs &a, const int32_t *n, const 
       g.act = m->x(); g.act_stride = dm.d; g.gain = m->attn_norm[l];
       g.out = m->qkv(); g.out_stride = dm.qkv_rows; g.out_col0 = 0;
       g.short_chain_row0 = prefill_t0 >= 0 ? nq : 0;   // a prompt's K and V rows: see launch_gemm_tc
+      g.out_is_zero = qkv_cleared ? 1 : 0;
       { ProfScope ps(m, PK_QKV); launches += project(m, g, EPI_STORE, ml); }
-      g.short_chain_row0 = 0;
+      g.short_chain_row0 = 0; g.out_is_zero = 0; qkv_cleared = false;
       { ProfScope ps(m, PK_ROPE);
         launches += launch_rope_append(m->qkv(), m->rope(), m->Kc, m->Vc, m->sched(), l, ROWS_PREFIX,
                                        0, ml, dm, st); }
@@ -341,7 +349,13 @@ static int32_t run_step(d3_model *m, const StepArgs &a, const int32_t *n, const 
       g.W = m->w_down[l]; g.W2 = nullptr; g.R = dm.d; g.K = dm.f; g.act = m->u();
       g.tmap_w = tm ? &m->tm_down[l] : nullptr; g.tmap_w2 = nullptr;
       g.act_stride = dm.f; g.gain = nullptr; g.out = m->x(); g.out_stride = dm.d;
+      if (clear_ahead) {
+        bool more = false;
+        for (int l2 = l + 1; l2 < L; ++l2) more = more || m_l[l2] > 0;
+        if (more) { g.clear = m->qkv(); g.clear_floats = (size_t)B * dm.qkv_rows; qkv_cleared = true; }
+      }
       { ProfScope ps(m, PK_DOWN); launches += project(m, g, EPI_RESID, ml); }
+      g.clear = nullptr; g.clear_floats = 0;
     }
     if (probe && logits_dev && l + 1 < L) {
       // every row's state after block l through the final norm and the LM head (Sec. 3.2)

@@ -91,6 +91,8 @@ struct TcArgs {
   int short_row0, chain_kb;
   int n_stages, tmem_cols;
   int atomic;            // combine with red.add (split-K or residual)
+  float4 *clear;         // nullable: a region for a later kernel, zeroed by the epilogue warps up front
+  unsigned clear_n4;     // its length in 16-byte units
   float *out;
   int out_stride, out_col0;
   const DevSched *sched;
@@ -351,6 +353,11 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
     // this call returns at once, and what this thread reads below (the schedule) is what they wrote
     bar_wait(smem_addr(&s_full[0]), 0u, abort_flag, t.wait_ns, true);
     pdl_wait();
+    if (t.clear) {   // nothing reads the region any more (the earlier kernels are complete)
+      const unsigned nthr = gridDim.x * gridDim.y * 128u;
+      for (unsigned i = (blockIdx.y * gridDim.x + blockIdx.x) * 128u + (unsigned)(tid - 64); i < t.clear_n4; i += nthr)
+        t.clear[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+    }
     int r0, r1;
     row_span(t.sched, t.layer, t.row_mode, r0, r1);
     const int nrows = min(r1 - r0, G * t.NP);
@@ -659,7 +666,7 @@ int launch_gemm_tc(TcContext &tc, const GemvArgs &g, int epi, int m_rows, cudaSt
   sa.act = g.act; sa.act_stride = g.act_stride; sa.K = g.K; sa.NP = NP; sa.N = N; sa.groups = groups;
   sa.gain = g.gain; sa.eps = g.eps;
   sa.dst = tc.act_split;
-  sa.zero_out = (epi == EPI_STORE && ksplit > 1) ? g.out : nullptr;
+  sa.zero_out = (epi == EPI_STORE && ksplit > 1 && !g.out_is_zero) ? g.out : nullptr;
   sa.out_stride = g.out_stride; sa.out_col0 = g.out_col0; sa.R = g.R;
   sa.sched = g.sched; sa.layer = g.layer; sa.row_mode = g.row_mode;
   launch_pdl(k_act_split, dim3(m_rows, (g.K + 1023) / 1024), dim3(256), 0, st, sa);
@@ -677,6 +684,7 @@ int launch_gemm_tc(TcContext &tc, const GemvArgs &g, int epi, int m_rows, cudaSt
   t.tmem_cols = 32;
   while (t.tmem_cols < groups * N) t.tmem_cols *= 2;
   t.atomic = (epi == EPI_RESID || (epi == EPI_STORE && ksplit > 1)) ? 1 : 0;
+  t.clear = reinterpret_cast<float4 *>(g.clear); t.clear_n4 = g.clear ? (unsigned)(g.clear_floats / 4) : 0u;
   t.out = g.out; t.out_stride = g.out_stride; t.out_col0 = g.out_col0;
   t.sched = g.sched; t.status = const_cast<DevSched *>(g.sched); t.layer = g.layer; t.row_mode = g.row_mode;
   t.wait_ns = tc.wait_ns;

@@ -72,6 +72,13 @@ struct GemvArgs {
   float *out;
   int out_stride;
   int out_col0;         // column offset added to the output row index r
+  // tensor-core path: `clear` (nullable) is a region of `clear_floats` floats (a multiple of 4, 16-byte
+  // aligned) that a LATER kernel wants zeroed and nothing reads any more: the projection's idle
+  // warps clear it while the weights stream.  `out_is_zero`: an earlier kernel did that for this
+  // projection's output rows, so the pre-pass of a split-K store need not.
+  float *clear;
+  size_t clear_floats;
+  int out_is_zero;
   int short_chain_row0; // tensor-core path: rows r >= this are summed in short slices (0 = off)
   const DevSched *sched;
   int layer;
