@@ -320,10 +320,13 @@ static int32_t run_step(d3_model *m, const StepArgs &a, const int32_t *n, const 
         if (len > max_len) max_len = len;
       }
       int ctas = ml * (dm.Hq / GQ);
-      static const int target_ctas = [] {   // tuning knob: pieces the attention pass aims for
+      // Pieces the attention pass aims for: one per SM.  More, shorter pieces lose to their fixed
+      // cost and to the combine pass (13B shape, 8 rows x 40 heads, 1024 positions: 6.13 ms per step
+      // with one piece per row and head, 6.30 with two; 70B shape, 4 rows: 24.2 against 24.5 ms).
+      static const int target_ctas = [] {   // tuning knob
         const char *env = getenv("D3_ATTN_TARGET_CTAS");
         const int v = env ? atoi(env) : 0;
-        return v >= 148 && v <= 65536 ? v : 592;
+        return v >= 32 && v <= 65536 ? v : 148;
       }();
       int want = (target_ctas + ctas - 1) / ctas;
       if (want < 1) want = 1;
