@@ -39,6 +39,7 @@ Layout make_layout(const d3_config &c) {
   if ((size_t)c.d_ffn > kmax) kmax = (size_t)c.d_ffn;
   y.act_split = off = align_up(off, 1024);
   y.act_split_bytes = (3 * ((B + 7) / 8 * 8) + 8) * kmax * sizeof(bf16);
+  y.act_split2 = off = align_up(off + y.act_split_bytes, 1024);
   off = align_up(off + y.act_split_bytes, 256);
   y.block_table = off;
   if (c.kv_layout == D3_KV_PAGED)
@@ -283,7 +284,7 @@ static int32_t run_step(d3_model *m, const StepArgs &a, const int32_t *n, const 
   memset(&g, 0, sizeof(g));
   g.sched = m->sched();
   g.eps = c.rms_eps;
-  g.clear = nullptr; g.clear_floats = 0; g.out_is_zero = 0;
+  g.clear = nullptr; g.clear_floats = 0; g.out_is_zero = 0; g.operand_out = g.operand_in = 0;
   // The QKV projection sums its k-slices into a zeroed buffer.  After a block's attention nothing
   // reads that buffer until the next block's projection, so the down projection in between clears
   // it on the side (decode steps without recomputed fills, which use the buffer in between).
@@ -347,7 +348,9 @@ static int32_t run_step(d3_model *m, const StepArgs &a, const int32_t *n, const 
       g.W = m->w_gate[l]; g.W2 = m->w_up[l]; g.R = dm.f; g.K = dm.d; g.act = m->x();
       g.tmap_w = tm ? &m->tm_gate[l] : nullptr; g.tmap_w2 = tm ? &m->tm_up[l] : nullptr;
       g.act_stride = dm.d; g.gain = m->mlp_norm[l]; g.out = m->u(); g.out_stride = dm.f;
+      g.operand_out = 1; m->tc.handed_over = false;
       { ProfScope ps(m, PK_GATEUP); launches += project(m, g, EPI_SWIGLU, ml); }
+      g.operand_out = 0;
       // down projection + residual
       g.W = m->w_down[l]; g.W2 = nullptr; g.R = dm.d; g.K = dm.f; g.act = m->u();
       g.tmap_w = tm ? &m->tm_down[l] : nullptr; g.tmap_w2 = nullptr;
@@ -357,8 +360,9 @@ static int32_t run_step(d3_model *m, const StepArgs &a, const int32_t *n, const 
         for (int l2 = l + 1; l2 < L; ++l2) more = more || m_l[l2] > 0;
         if (more) { g.clear = m->qkv(); g.clear_floats = (size_t)B * dm.qkv_rows; qkv_cleared = true; }
       }
+      g.operand_in = m->tc.handed_over ? 1 : 0;
       { ProfScope ps(m, PK_DOWN); launches += project(m, g, EPI_RESID, ml); }
-      g.clear = nullptr; g.clear_floats = 0;
+      g.clear = nullptr; g.clear_floats = 0; g.operand_in = 0; m->tc.handed_over = false;
     }
     if (probe && logits_dev && l + 1 < L) {
       // every row's state after block l through the final norm and the LM head (Sec. 3.2)
@@ -612,6 +616,8 @@ int32_t d3_load(const d3_config *cfg, const d3_weights *w, void *kv_dev, void *s
   // tensor-core projections: usable when the driver encodes every weight's tensor map
   m->tc.ok = tc_init() == 0;
   m->tc.act_split = reinterpret_cast<bf16 *>(m->scratch + m->lay.act_split);
+  m->tc.act_split2 = reinterpret_cast<bf16 *>(m->scratch + m->lay.act_split2);
+  m->tc.handed_over = false;
   m->tc.act_bytes = m->lay.act_split_bytes;
   m->wait_ns = 2000000000ull;
   m->stall_next = 0;

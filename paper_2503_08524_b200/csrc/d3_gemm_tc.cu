@@ -91,6 +91,7 @@ struct TcArgs {
   int short_row0, chain_kb;
   int n_stages, tmem_cols;
   int atomic;            // combine with red.add (split-K or residual)
+  bf16 *opnd_out;        // nullable (SiLU * mul epilogue): the result also as the next projection's operand, [3 NP][R]
   float4 *clear;         // nullable: a region for a later kernel, zeroed by the epilogue warps up front
   unsigned clear_n4;     // its length in 16-byte units
   float *out;
@@ -439,7 +440,16 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CU
             const int j = j0 + i;
             if (j < nrows && r < t.R) {
               const float z = y[i], up = xch[j * kBoxRows + trow];
-              t.out[(size_t)(r0 + j) * t.out_stride + t.out_col0 + r] = z / (1.f + __expf(-z)) * up;
+              const float val = z / (1.f + __expf(-z)) * up;
+              t.out[(size_t)(r0 + j) * t.out_stride + t.out_col0 + r] = val;
+              if (t.opnd_out) {   // hi + mid + lo = val, rows j, NP + j, 2 NP + j of the next operand
+                const bf16 h = __float2bfloat16_rn(val);
+                const float r1 = val - __bfloat162float(h);     // exact
+                const bf16 md = __float2bfloat16_rn(r1);
+                const bf16 lw = __float2bfloat16_rn(r1 - __bfloat162float(md));
+                bf16 *o = t.opnd_out + (size_t)j * t.R + r;
+                o[0] = h; o[(size_t)t.NP * t.R] = md; o[(size_t)2 * t.NP * t.R] = lw;
+              }
             }
           }
         }
@@ -624,11 +634,13 @@ int launch_gemm_tc(TcContext &tc, const GemvArgs &g, int epi, int m_rows, cudaSt
   const int groups = m_rows > kGroupRows ? 2 : 1;
   const int NP = groups > 1 ? kGroupRows : (m_rows + 7) / 8 * 8, N = (3 * NP + 15) / 16 * 16;
   if ((size_t)groups * N * g.K * sizeof(bf16) > tc.act_bytes) return 0;
-  const uint64_t key = ((uint64_t)groups << 48) | ((uint64_t)NP << 32) | (uint32_t)g.K;
+  // the operand comes from the pre-pass (act_split) or was left by the previous projection (act_split2)
+  const bool handed = g.operand_in && groups == 1 && !g.gain && epi == EPI_RESID;
+  const uint64_t key = ((uint64_t)(handed ? 1 : 0) << 56) | ((uint64_t)groups << 48) | ((uint64_t)NP << 32) | (uint32_t)g.K;
   auto it = tc.act_maps.find(key);
   if (it == tc.act_maps.end()) {
     TMap mp;
-    if (!encode_map(&mp, tc.act_split, groups * N, g.K, N)) return 0;
+    if (!encode_map(&mp, handed ? tc.act_split2 : tc.act_split, groups * N, g.K, N)) return 0;
     it = tc.act_maps.emplace(key, mp).first;
   }
 
@@ -669,7 +681,7 @@ int launch_gemm_tc(TcContext &tc, const GemvArgs &g, int epi, int m_rows, cudaSt
   sa.zero_out = (epi == EPI_STORE && ksplit > 1 && !g.out_is_zero) ? g.out : nullptr;
   sa.out_stride = g.out_stride; sa.out_col0 = g.out_col0; sa.R = g.R;
   sa.sched = g.sched; sa.layer = g.layer; sa.row_mode = g.row_mode;
-  launch_pdl(k_act_split, dim3(m_rows, (g.K + 1023) / 1024), dim3(256), 0, st, sa);
+  if (!handed) launch_pdl(k_act_split, dim3(m_rows, (g.K + 1023) / 1024), dim3(256), 0, st, sa);
 
   TcArgs t;
   t.R = g.R; t.K = g.K; t.NP = NP; t.N = N; t.groups = groups; t.n_kb = n_kb; t.kb_per_split = per;
@@ -684,6 +696,11 @@ int launch_gemm_tc(TcContext &tc, const GemvArgs &g, int epi, int m_rows, cudaSt
   t.tmem_cols = 32;
   while (t.tmem_cols < groups * N) t.tmem_cols *= 2;
   t.atomic = (epi == EPI_RESID || (epi == EPI_STORE && ksplit > 1)) ? 1 : 0;
+  t.opnd_out = nullptr;
+  if (g.operand_out && epi == EPI_SWIGLU && groups == 1 && (size_t)N * g.R * sizeof(bf16) <= tc.act_bytes && g.R % 8 == 0) {
+    t.opnd_out = tc.act_split2;
+    tc.handed_over = true;
+  }
   t.clear = reinterpret_cast<float4 *>(g.clear); t.clear_n4 = g.clear ? (unsigned)(g.clear_floats / 4) : 0u;
   t.out = g.out; t.out_stride = g.out_stride; t.out_col0 = g.out_col0;
   t.sched = g.sched; t.status = const_cast<DevSched *>(g.sched); t.layer = g.layer; t.row_mode = g.row_mode;
@@ -702,7 +719,7 @@ int launch_gemm_tc(TcContext &tc, const GemvArgs &g, int epi, int m_rows, cudaSt
     case EPI_SWIGLU: launch_pdl(k_gemm_tc<EPI_SWIGLU>, grid, dim3(kTcThreads), smem, st, *w0, *w1, *ma, t); break;
     default: launch_pdl(k_gemm_tc<EPI_LOGITS>, grid, dim3(kTcThreads), smem, st, *w0, *w1, *ma, t); break;
   }
-  return 2;
+  return handed ? 1 : 2;
 }
 
 }  // namespace d3

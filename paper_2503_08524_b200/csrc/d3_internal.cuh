@@ -79,6 +79,10 @@ struct GemvArgs {
   float *clear;
   size_t clear_floats;
   int out_is_zero;
+  // tensor-core path, operand hand-over between two projections of the same rows (<= 64):
+  // `operand_out`: the SiLU * mul epilogue also writes its result as the three-term bf16 operand of
+  // the projection that follows; `operand_in`: that operand is there, no pre-pass runs.
+  int operand_out, operand_in;
   int short_chain_row0; // tensor-core path: rows r >= this are summed in short slices (0 = off)
   const DevSched *sched;
   int layer;
@@ -143,6 +147,8 @@ static constexpr unsigned long long kDrainFloorNs = 1000000ull;
 struct TcContext {
   bool ok;                              // the driver's tensor-map encoder is there and the kernels are set up
   bf16 *act_split;                      // device: activations as bf16 hi, mid, lo rows, [3 NP][K]
+  bf16 *act_split2;                     // a second one, written by a projection's epilogue for the next
+  bool handed_over;                     // the last launch wrote act_split2 (GemvArgs.operand_out honoured)
   size_t act_bytes;
   std::map<uint64_t, TMap> act_maps;    // tensor maps of act_split, keyed by (NP, K)
   int sm_count;
@@ -152,7 +158,7 @@ struct TcContext {
 // Byte offsets of the regions of the caller's scratch buffer.
 struct Layout {
   size_t sched, rope, x, qkv, attn_out, part_o, part_ml, u, layer_tab, bar, phase, part_fused, act_split,
-      act_split_bytes, block_table, total;
+      act_split2, act_split_bytes, block_table, total;
   int max_splits;
 };
 
