@@ -305,6 +305,7 @@ static int32_t run_step(d3_model *m, const StepArgs &a, const int32_t *n, const 
       g.out_is_zero = qkv_cleared ? 1 : 0;
       { ProfScope ps(m, PK_QKV); launches += project(m, g, EPI_STORE, ml); }
       g.short_chain_row0 = 0; g.out_is_zero = 0; qkv_cleared = false;
+      bool o_handed = false;
       { ProfScope ps(m, PK_ROPE);
         launches += launch_rope_append(m->qkv(), m->rope(), m->Kc, m->Vc, m->sched(), l, ROWS_PREFIX,
                                        0, ml, dm, st); }
@@ -336,14 +337,20 @@ static int32_t run_step(d3_model *m, const StepArgs &a, const int32_t *n, const 
       if (split_len < 32) split_len = 32;
       int n_splits = (max_len + split_len - 1) / split_len;
       { ProfScope ps(m, PK_ATTN);
+        // the output projection's three-term operand, when that projection will go to the tensor cores
+        OpndOut opnd = {nullptr, 0};
+        const bool tensor = m->exec_mode == D3_EXEC_TENSOR || (m->exec_mode == D3_EXEC_AUTO && ml >= D3_TENSOR_MIN_ROWS);
+        if (tensor && m->tm_ok && ml <= 64) { opnd.p = m->tc.act_split2; opnd.np = (ml + 7) / 8 * 8; o_handed = true; }
         launches += launch_attention(m->qkv(), m->Kc, m->Vc, m->sched(), l, ml, split_len, n_splits,
-                                     m->lay.max_splits, m->part_o(), m->part_ml(), m->attn_out(), dm, st); }
+                                     m->lay.max_splits, m->part_o(), m->part_ml(), m->attn_out(), opnd, dm, st); }
       }
       // output projection + residual
       g.W = m->wo[l]; g.R = dm.d; g.K = nq; g.act = m->attn_out(); g.act_stride = nq;
       g.tmap_w = tm ? &m->tm_o[l] : nullptr;
       g.gain = nullptr; g.out = m->x(); g.out_stride = dm.d;
+      g.operand_in = o_handed ? 1 : 0;
       { ProfScope ps(m, PK_OPROJ); launches += project(m, g, EPI_RESID, ml); }
+      g.operand_in = 0;
       // RMSNorm + gate/up + SiLU * mul
       g.W = m->w_gate[l]; g.W2 = m->w_up[l]; g.R = dm.f; g.K = dm.d; g.act = m->x();
       g.tmap_w = tm ? &m->tm_gate[l] : nullptr; g.tmap_w2 = tm ? &m->tm_up[l] : nullptr;

@@ -52,7 +52,8 @@ struct VStage {
 template <int DH, int GQ>
 __global__ void __launch_bounds__(kAThreads)
 k_attn_partial_mma(const float *qkv, const bf16 *Kc, const bf16 *Vc, const DevSched *s, int layer,
-                   int split_len, int max_splits, float *part_o, float *part_ml, float *attn_out, Dims dm) {
+                   int split_len, int max_splits, float *part_o, float *part_ml, float *attn_out, OpndOut opnd,
+                   Dims dm) {
   static_assert(GQ <= 8, "one accumulator row per query head");
   constexpr int KK = DH / 16;          // MMA steps over the head dimension
   constexpr int NT = DH / 8;           // 8-wide dimension tiles of the output
@@ -221,7 +222,9 @@ k_attn_partial_mma(const float *qkv, const bf16 *Kc, const bf16 *Vc, const DevSc
       O += s_o[w][gg][e] * c;
     }
     if (attn_out) {   // the only piece of its row and head: the result itself, no combine pass
-      attn_out[(size_t)row * dm.Hq * DH + (size_t)(h0 + gg) * DH + e] = O / Lsum;
+      const float val = O / Lsum;
+      attn_out[(size_t)row * dm.Hq * DH + (size_t)(h0 + gg) * DH + e] = val;
+      if (opnd.p) opnd_store(opnd, row, (size_t)dm.Hq * DH, (size_t)(h0 + gg) * DH + e, val);
       continue;
     }
     const size_t pi = ((size_t)row * dm.Hq + h0 + gg) * max_splits + split;
@@ -242,17 +245,17 @@ cudaError_t mma_attr() {
 template <int DH>
 void launch_dh(const float *qkv, const bf16 *Kc, const bf16 *Vc, const DevSched *s, int layer, int m_rows,
                int split_len, int n_splits, int max_splits, float *part_o, float *part_ml, float *attn_out,
-               const Dims &dm, cudaStream_t st) {
+               OpndOut opnd, const Dims &dm, cudaStream_t st) {
   const int G = dm.Hq / dm.Hkv;
   if (G % 4 == 0) {
     launch_pdl(k_attn_partial_mma<DH, 4>, dim3(n_splits, dm.Hq / 4, m_rows), dim3(kAThreads), v_smem<DH>(), st,
-               qkv, Kc, Vc, s, layer, split_len, max_splits, part_o, part_ml, attn_out, dm);
+               qkv, Kc, Vc, s, layer, split_len, max_splits, part_o, part_ml, attn_out, opnd, dm);
   } else if (G % 2 == 0) {
     launch_pdl(k_attn_partial_mma<DH, 2>, dim3(n_splits, dm.Hq / 2, m_rows), dim3(kAThreads), v_smem<DH>(), st,
-               qkv, Kc, Vc, s, layer, split_len, max_splits, part_o, part_ml, attn_out, dm);
+               qkv, Kc, Vc, s, layer, split_len, max_splits, part_o, part_ml, attn_out, opnd, dm);
   } else {
     launch_pdl(k_attn_partial_mma<DH, 1>, dim3(n_splits, dm.Hq, m_rows), dim3(kAThreads), v_smem<DH>(), st,
-               qkv, Kc, Vc, s, layer, split_len, max_splits, part_o, part_ml, attn_out, dm);
+               qkv, Kc, Vc, s, layer, split_len, max_splits, part_o, part_ml, attn_out, opnd, dm);
   }
 }
 
@@ -273,13 +276,13 @@ int init_attention_mma() {
 // piece per row and head): the normalised result goes there and no combine pass is needed.
 int launch_attention_partial_mma(const float *qkv, const bf16 *Kc, const bf16 *Vc, const DevSched *s, int layer,
                                  int m_rows, int split_len, int n_splits, int max_splits, float *part_o,
-                                 float *part_ml, float *attn_out, const Dims &dm, cudaStream_t st) {
+                                 float *part_ml, float *attn_out, OpndOut opnd, const Dims &dm, cudaStream_t st) {
   if (dm.dh == 128)
-    launch_dh<128>(qkv, Kc, Vc, s, layer, m_rows, split_len, n_splits, max_splits, part_o, part_ml, attn_out, dm, st);
+    launch_dh<128>(qkv, Kc, Vc, s, layer, m_rows, split_len, n_splits, max_splits, part_o, part_ml, attn_out, opnd, dm, st);
   else if (dm.dh == 64)
-    launch_dh<64>(qkv, Kc, Vc, s, layer, m_rows, split_len, n_splits, max_splits, part_o, part_ml, attn_out, dm, st);
+    launch_dh<64>(qkv, Kc, Vc, s, layer, m_rows, split_len, n_splits, max_splits, part_o, part_ml, attn_out, opnd, dm, st);
   else
-    launch_dh<32>(qkv, Kc, Vc, s, layer, m_rows, split_len, n_splits, max_splits, part_o, part_ml, attn_out, dm, st);
+    launch_dh<32>(qkv, Kc, Vc, s, layer, m_rows, split_len, n_splits, max_splits, part_o, part_ml, attn_out, opnd, dm, st);
   return 1;
 }
 

@@ -61,6 +61,10 @@ struct alignas(64) TMap {
   uint64_t w[16];
 };
 
+// Where a kernel also leaves its fp32 result as the three-term bf16 operand of the tensor-core
+// projection that follows (rows j, np + j, 2 np + j of [3 np][K]); p == nullptr: nowhere.
+struct OpndOut { bf16 *p; int np; };
+
 struct GemvArgs {
   const bf16 *W, *W2;   // [R][K] row-major (W2: second matrix of EPI_SWIGLU)
   const TMap *tmap_w, *tmap_w2;  // host pointers, nullable: tensor maps of W and W2 (tensor-core path)
@@ -174,6 +178,15 @@ struct Layout {
 #ifdef __CUDACC__
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+// v as the three bf16 terms hi + mid + lo of row j of a projection operand [3 np][K]
+__device__ __forceinline__ void opnd_store(const OpndOut &o, int j, size_t K, size_t col, float v) {
+  const bf16 h = __float2bfloat16_rn(v);
+  const float r1 = v - __bfloat162float(h);     // exact
+  const bf16 md = __float2bfloat16_rn(r1);
+  const bf16 lw = __float2bfloat16_rn(r1 - __bfloat162float(md));
+  bf16 *p = o.p + (size_t)j * K + col;
+  p[0] = h; p[(size_t)o.np * K] = md; p[(size_t)2 * o.np * K] = lw;
+}
 
 template <typename... KArgs, typename... Args>
 inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
@@ -209,14 +222,14 @@ int launch_rope_append(float *qkv, const float2 *rope, bf16 *Kc, bf16 *Vc, const
                        cudaStream_t st);
 int launch_attention(const float *qkv, const bf16 *Kc, const bf16 *Vc, const DevSched *s, int layer,
                      int m_rows, int split_len, int n_splits, int max_splits, float *part_o,
-                     float *part_ml, float *attn_out, const Dims &dm, cudaStream_t st);
+                     float *part_ml, float *attn_out, OpndOut opnd, const Dims &dm, cudaStream_t st);
 int init_attention_mma();
 int init_attention_prefill();
 int launch_attention_prefill(const float *qkv, const bf16 *Kc, const bf16 *Vc, int layer, int slot, int t0, int B,
                              float *attn_out, const Dims &dm, cudaStream_t st);
 int launch_attention_partial_mma(const float *qkv, const bf16 *Kc, const bf16 *Vc, const DevSched *s, int layer,
                                  int m_rows, int split_len, int n_splits, int max_splits, float *part_o,
-                                 float *part_ml, float *attn_out, const Dims &dm, cudaStream_t st);
+                                 float *part_ml, float *attn_out, OpndOut opnd, const Dims &dm, cudaStream_t st);
 int launch_fill_copy(bf16 *Kc, bf16 *Vc, const DevSched *s, int B, const Dims &dm, cudaStream_t st);
 int launch_argmax(const float *logits, int B, int V, int32_t *out, cudaStream_t st);
 int launch_argmax_conf(const float *logits, int B, int V, int32_t *tok, float *conf, int stride, int col,

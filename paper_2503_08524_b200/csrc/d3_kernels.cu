@@ -522,7 +522,7 @@ k_attn_partial(const float *qkv, const bf16 *Kc, const bf16 *Vc, const DevSched 
 
 // merge the splits of one (row, head): attn_out[row][h*dh + e]
 __global__ void k_attn_combine(const float *part_o, const float *part_ml, const DevSched *s, int layer,
-                               int split_len, int max_splits, float *attn_out, Dims dm) {
+                               int split_len, int max_splits, float *attn_out, OpndOut opnd, Dims dm) {
   pdl_wait();
   pdl_trigger();
   const int row = blockIdx.y, h = blockIdx.x, e = threadIdx.x;
@@ -538,7 +538,9 @@ __global__ void k_attn_combine(const float *part_o, const float *part_ml, const 
     Lsum += part_ml[(pi + i) * 2 + 1] * c;
     O += part_o[(pi + i) * dm.dh + e] * c;
   }
-  attn_out[(size_t)row * dm.Hq * dm.dh + h * dm.dh + e] = O / Lsum;
+  const float val = O / Lsum;
+  attn_out[(size_t)row * dm.Hq * dm.dh + h * dm.dh + e] = val;
+  if (opnd.p) opnd_store(opnd, row, (size_t)dm.Hq * dm.dh, (size_t)h * dm.dh + e, val);
 }
 
 template <int DH>
@@ -563,7 +565,7 @@ static void attn_launch(const float *qkv, const bf16 *Kc, const bf16 *Vc, const 
 
 int launch_attention(const float *qkv, const bf16 *Kc, const bf16 *Vc, const DevSched *s, int layer,
                      int m_rows, int split_len, int n_splits, int max_splits, float *part_o,
-                     float *part_ml, float *attn_out, const Dims &dm, cudaStream_t st) {
+                     float *part_ml, float *attn_out, OpndOut opnd, const Dims &dm, cudaStream_t st) {
   static const bool fma_path = getenv("D3_ATTN_FMA") != nullptr;   // the scalar kernel, for comparison
   // The tensor-core kernel pays a fixed cost per CTA (Q fragments, merge) that needs a few
   // 16-position trips per warp to amortise, unless several query heads share the K/V fragments:
@@ -571,7 +573,7 @@ int launch_attention(const float *qkv, const bf16 *Kc, const bf16 *Vc, const Dev
   const bool shared_kv = (dm.Hq / dm.Hkv) % 2 == 0;
   if (!fma_path && (shared_kv || split_len >= 256)) {
     launch_attention_partial_mma(qkv, Kc, Vc, s, layer, m_rows, split_len, n_splits, max_splits, part_o,
-                                 part_ml, n_splits == 1 ? attn_out : nullptr, dm, st);
+                                 part_ml, n_splits == 1 ? attn_out : nullptr, opnd, dm, st);
     if (n_splits == 1) return 1;   // every row and head in one piece: written directly
   } else if (dm.dh == 128)
     attn_launch<128>(qkv, Kc, Vc, s, layer, m_rows, split_len, n_splits, max_splits, part_o, part_ml, dm, st);
@@ -581,7 +583,7 @@ int launch_attention(const float *qkv, const bf16 *Kc, const bf16 *Vc, const Dev
     attn_launch<32>(qkv, Kc, Vc, s, layer, m_rows, split_len, n_splits, max_splits, part_o, part_ml, dm, st);
   dim3 cgrid(dm.Hq, m_rows);
   launch_pdl(k_attn_combine, cgrid, dim3(dm.dh), 0, st, part_o, part_ml, s, layer, split_len, max_splits,
-             attn_out, dm);
+             attn_out, opnd, dm);
   return 2;
 }
 
