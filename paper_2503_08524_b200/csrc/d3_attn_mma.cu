@@ -53,7 +53,7 @@ template <int DH, int GQ>
 __global__ void __launch_bounds__(kAThreads)
 k_attn_partial_mma(const float *qkv, const bf16 *Kc, const bf16 *Vc, const DevSched *s, int layer,
                    int split_len, int max_splits, float *part_o, float *part_ml, float *attn_out, OpndOut opnd,
-                   Dims dm) {
+                   Dims dm, const __grid_constant__ RowOrder order) {
   static_assert(GQ <= 8, "one accumulator row per query head");
   constexpr int KK = DH / 16;          // MMA steps over the head dimension
   constexpr int NT = DH / 8;           // 8-wide dimension tiles of the output
@@ -62,7 +62,7 @@ k_attn_partial_mma(const float *qkv, const bf16 *Kc, const bf16 *Vc, const DevSc
   __shared__ float s_m[kAWarps][GQ], s_l[kAWarps][GQ];
   pdl_wait();
   pdl_trigger();
-  const int row = blockIdx.z;
+  const int row = order.given ? order.r[blockIdx.z] : blockIdx.z;
   if (row >= s->m[layer]) return;
   const int len = s->pos_s[row] + 1;
   const int split = blockIdx.x;
@@ -245,17 +245,17 @@ cudaError_t mma_attr() {
 template <int DH>
 void launch_dh(const float *qkv, const bf16 *Kc, const bf16 *Vc, const DevSched *s, int layer, int m_rows,
                int split_len, int n_splits, int max_splits, float *part_o, float *part_ml, float *attn_out,
-               OpndOut opnd, const Dims &dm, cudaStream_t st) {
+               OpndOut opnd, const Dims &dm, cudaStream_t st, const RowOrder &order) {
   const int G = dm.Hq / dm.Hkv;
   if (G % 4 == 0) {
     launch_pdl(k_attn_partial_mma<DH, 4>, dim3(n_splits, dm.Hq / 4, m_rows), dim3(kAThreads), v_smem<DH>(), st,
-               qkv, Kc, Vc, s, layer, split_len, max_splits, part_o, part_ml, attn_out, opnd, dm);
+               qkv, Kc, Vc, s, layer, split_len, max_splits, part_o, part_ml, attn_out, opnd, dm, order);
   } else if (G % 2 == 0) {
     launch_pdl(k_attn_partial_mma<DH, 2>, dim3(n_splits, dm.Hq / 2, m_rows), dim3(kAThreads), v_smem<DH>(), st,
-               qkv, Kc, Vc, s, layer, split_len, max_splits, part_o, part_ml, attn_out, opnd, dm);
+               qkv, Kc, Vc, s, layer, split_len, max_splits, part_o, part_ml, attn_out, opnd, dm, order);
   } else {
     launch_pdl(k_attn_partial_mma<DH, 1>, dim3(n_splits, dm.Hq, m_rows), dim3(kAThreads), v_smem<DH>(), st,
-               qkv, Kc, Vc, s, layer, split_len, max_splits, part_o, part_ml, attn_out, opnd, dm);
+               qkv, Kc, Vc, s, layer, split_len, max_splits, part_o, part_ml, attn_out, opnd, dm, order);
   }
 }
 
@@ -276,13 +276,16 @@ int init_attention_mma() {
 // piece per row and head): the normalised result goes there and no combine pass is needed.
 int launch_attention_partial_mma(const float *qkv, const bf16 *Kc, const bf16 *Vc, const DevSched *s, int layer,
                                  int m_rows, int split_len, int n_splits, int max_splits, float *part_o,
-                                 float *part_ml, float *attn_out, OpndOut opnd, const Dims &dm, cudaStream_t st) {
+                                 float *part_ml, float *attn_out, OpndOut opnd, const Dims &dm, cudaStream_t st,
+                                 const RowOrder *order_in) {
+  RowOrder order;
+  if (order_in) order = *order_in; else order.given = 0;
   if (dm.dh == 128)
-    launch_dh<128>(qkv, Kc, Vc, s, layer, m_rows, split_len, n_splits, max_splits, part_o, part_ml, attn_out, opnd, dm, st);
+    launch_dh<128>(qkv, Kc, Vc, s, layer, m_rows, split_len, n_splits, max_splits, part_o, part_ml, attn_out, opnd, dm, st, order);
   else if (dm.dh == 64)
-    launch_dh<64>(qkv, Kc, Vc, s, layer, m_rows, split_len, n_splits, max_splits, part_o, part_ml, attn_out, opnd, dm, st);
+    launch_dh<64>(qkv, Kc, Vc, s, layer, m_rows, split_len, n_splits, max_splits, part_o, part_ml, attn_out, opnd, dm, st, order);
   else
-    launch_dh<32>(qkv, Kc, Vc, s, layer, m_rows, split_len, n_splits, max_splits, part_o, part_ml, attn_out, opnd, dm, st);
+    launch_dh<32>(qkv, Kc, Vc, s, layer, m_rows, split_len, n_splits, max_splits, part_o, part_ml, attn_out, opnd, dm, st, order);
   return 1;
 }
 

@@ -64,6 +64,9 @@ struct alignas(64) TMap {
 // Where a kernel also leaves its fp32 result as the three-term bf16 operand of the tensor-core
 // projection that follows (rows j, np + j, 2 np + j of [3 np][K]); p == nullptr: nowhere.
 struct OpndOut { bf16 *p; int np; };
+// The order in which an attention launch takes the rows (longest context first, so that the short
+// ones fill the tail); given == 0: as they come.
+struct RowOrder { unsigned char r[D3_MAX_BATCH]; int given; };
 
 struct GemvArgs {
   const bf16 *W, *W2;   // [R][K] row-major (W2: second matrix of EPI_SWIGLU)
@@ -222,14 +225,16 @@ int launch_rope_append(float *qkv, const float2 *rope, bf16 *Kc, bf16 *Vc, const
                        cudaStream_t st);
 int launch_attention(const float *qkv, const bf16 *Kc, const bf16 *Vc, const DevSched *s, int layer,
                      int m_rows, int split_len, int n_splits, int max_splits, float *part_o,
-                     float *part_ml, float *attn_out, OpndOut opnd, const Dims &dm, cudaStream_t st);
+                     float *part_ml, float *attn_out, OpndOut opnd, const Dims &dm, cudaStream_t st,
+                     const RowOrder *order = nullptr);
 int init_attention_mma();
 int init_attention_prefill();
 int launch_attention_prefill(const float *qkv, const bf16 *Kc, const bf16 *Vc, int layer, int slot, int t0, int B,
                              float *attn_out, const Dims &dm, cudaStream_t st);
 int launch_attention_partial_mma(const float *qkv, const bf16 *Kc, const bf16 *Vc, const DevSched *s, int layer,
                                  int m_rows, int split_len, int n_splits, int max_splits, float *part_o,
-                                 float *part_ml, float *attn_out, OpndOut opnd, const Dims &dm, cudaStream_t st);
+                                 float *part_ml, float *attn_out, OpndOut opnd, const Dims &dm, cudaStream_t st,
+                                 const RowOrder *order = nullptr);
 int launch_fill_copy(bf16 *Kc, bf16 *Vc, const DevSched *s, int B, const Dims &dm, cudaStream_t st);
 int launch_argmax(const float *logits, int B, int V, int32_t *out, cudaStream_t st);
 int launch_argmax_conf(const float *logits, int B, int V, int32_t *tok, float *conf, int stride, int col,

@@ -565,7 +565,8 @@ static void attn_launch(const float *qkv, const bf16 *Kc, const bf16 *Vc, const 
 
 int launch_attention(const float *qkv, const bf16 *Kc, const bf16 *Vc, const DevSched *s, int layer,
                      int m_rows, int split_len, int n_splits, int max_splits, float *part_o,
-                     float *part_ml, float *attn_out, OpndOut opnd, const Dims &dm, cudaStream_t st) {
+                     float *part_ml, float *attn_out, OpndOut opnd, const Dims &dm, cudaStream_t st,
+                     const RowOrder *order) {
   static const bool fma_path = getenv("D3_ATTN_FMA") != nullptr;   // the scalar kernel, for comparison
   // The tensor-core kernel pays a fixed cost per CTA (Q fragments, merge) that needs a few
   // 16-position trips per warp to amortise, unless several query heads share the K/V fragments:
@@ -573,7 +574,7 @@ int launch_attention(const float *qkv, const bf16 *Kc, const bf16 *Vc, const Dev
   const bool shared_kv = (dm.Hq / dm.Hkv) % 2 == 0;
   if (!fma_path && (shared_kv || split_len >= 256)) {
     launch_attention_partial_mma(qkv, Kc, Vc, s, layer, m_rows, split_len, n_splits, max_splits, part_o,
-                                 part_ml, n_splits == 1 ? attn_out : nullptr, opnd, dm, st);
+                                 part_ml, n_splits == 1 ? attn_out : nullptr, opnd, dm, st, order);
     if (n_splits == 1) return 1;   // every row and head in one piece: written directly
   } else if (dm.dh == 128)
     attn_launch<128>(qkv, Kc, Vc, s, layer, m_rows, split_len, n_splits, max_splits, part_o, part_ml, dm, st);
