@@ -242,6 +242,12 @@ static int32_t pages_for_step(d3_model *m, int B, const int32_t *slot, const int
   return D3_OK;
 }
 
+// Up to this many rows the kernel in front of the O and down projections writes their three-term
+// operand itself (no pre-pass).  Measured on the 7B shape, ms per step with / without: 16 rows 3.60 /
+// 3.77, 32 rows 4.13 / 4.29, 40 rows 4.51 / 4.65, but 48 rows 6.0 / 5.35 and 56 rows 5.71 / 5.63: the
+// 2-byte stores of a wide group cost the epilogues more than the pre-passes they replace.
+static const int kHandOverMaxRows = 40;
+
 // One projection over `rows` rows: tensor cores for a dense enough group, FMA GEMV otherwise.
 static int project(d3_model *m, const GemvArgs &g, int epi, int rows) {
   const bool tensor = m->exec_mode == D3_EXEC_TENSOR ||
@@ -341,7 +347,7 @@ static int32_t run_step(d3_model *m, const StepArgs &a, const int32_t *n, const 
         // the output projection's three-term operand, when that projection will go to the tensor cores
         OpndOut opnd = {nullptr, 0};
         const bool tensor = m->exec_mode == D3_EXEC_TENSOR || (m->exec_mode == D3_EXEC_AUTO && ml >= D3_TENSOR_MIN_ROWS);
-        if (tensor && m->tm_ok && ml <= 64) { opnd.p = m->tc.act_split2; opnd.np = (ml + 7) / 8 * 8; o_handed = true; }
+        if (tensor && m->tm_ok && ml <= kHandOverMaxRows) { opnd.p = m->tc.act_split2; opnd.np = (ml + 7) / 8 * 8; o_handed = true; }
         // longest contexts first: the launch's last CTAs are then short ones (C3: 0.4 % of the step)
         RowOrder order;
         order.given = 1;
@@ -366,7 +372,7 @@ static int32_t run_step(d3_model *m, const StepArgs &a, const int32_t *n, const 
       g.W = m->w_gate[l]; g.W2 = m->w_up[l]; g.R = dm.f; g.K = dm.d; g.act = m->x();
       g.tmap_w = tm ? &m->tm_gate[l] : nullptr; g.tmap_w2 = tm ? &m->tm_up[l] : nullptr;
       g.act_stride = dm.d; g.gain = m->mlp_norm[l]; g.out = m->u(); g.out_stride = dm.f;
-      g.operand_out = 1; m->tc.handed_over = false;
+      g.operand_out = ml <= kHandOverMaxRows ? 1 : 0; m->tc.handed_over = false;
       { ProfScope ps(m, PK_GATEUP); launches += project(m, g, EPI_SWIGLU, ml); }
       g.operand_out = 0;
       // down projection + residual
